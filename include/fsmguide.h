@@ -1,0 +1,171 @@
+/*
+ * fsmguide - FSM vocabulary indexing and masked greedy decoding on NVIDIA B200
+ * (sm_100a), after "Efficient Guided Generation for Large Language Models"
+ * (arXiv 2307.09702).
+ *
+ * C ABI.  Unless an argument is marked HOST, every array pointer is a DEVICE
+ * pointer owned by the caller; the library neither allocates nor frees device
+ * memory, never synchronises the stream and never aborts.  All work is
+ * enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = the default
+ * stream) and may still be running when a call returns.
+ *
+ * Return value: FSM_OK, or a negative FSM_ERR_* code.  Errors that can be
+ * detected from the scalar arguments and pointer values are returned before
+ * anything is enqueued.  Faults in the *contents* of device arrays cannot be
+ * seen from the host without a synchronisation; kernels neutralise them (see
+ * each argument) and OR a FSM_FLAG_* bit into `*status_word`, a device int32
+ * the caller zeroes beforehand and may read after synchronising.  `status_word`
+ * may be NULL.
+ */
+#ifndef FSMGUIDE_H
+#define FSMGUIDE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FSM_OK 0
+#define FSM_ERR_NULL (-1)      /* a required pointer is NULL */
+#define FSM_ERR_SHAPE (-2)     /* a size is non-positive or inconsistent */
+#define FSM_ERR_ALIGN (-3)     /* a pointer or stride breaks the stated alignment */
+#define FSM_ERR_DTYPE (-4)     /* unknown dtype code, or FSM_STATE_U16 with Q > 65535 */
+#define FSM_ERR_WORKSPACE (-5) /* workspace missing or smaller than the query says */
+#define FSM_ERR_RANGE (-6)     /* dead_state, eos_id or a row range is out of range */
+#define FSM_ERR_CUDA (-7)      /* a CUDA runtime call failed (launch, attribute) */
+#define FSM_ERR_DEVICE (-8)    /* no device of compute capability 10.x is current */
+
+/* Bits of *status_word (device int32). */
+#define FSM_FLAG_TRANS_RANGE 1   /* a transition outside [0,Q) was read; treated as dead */
+#define FSM_FLAG_OFFSETS 2       /* vocab_offsets not non-decreasing / out of bounds; token
+                                    treated as empty */
+#define FSM_FLAG_STATE_RANGE 4   /* states[i] outside [0,Q); row finished as stuck */
+#define FSM_FLAG_CLASS_SPLIT 8   /* informational: two byte columns hashed alike but differ;
+                                    the build took the uncompressed path (still exact) */
+#define FSM_FLAG_WAIT_TIMEOUT 16 /* a bounded wait on an on-chip copy gave up; output invalid */
+
+typedef enum { FSM_STATE_I32 = 0, FSM_STATE_U16 = 1 } fsm_state_dtype;
+typedef enum { FSM_LOGITS_F32 = 0, FSM_LOGITS_BF16 = 1 } fsm_logits_dtype;
+
+/* Text for a return code ("FSM_OK", "FSM_ERR_NULL: ...").  HOST string, static. */
+const char* fsm_status_string(int status);
+
+/* FSM_OK if the current device has compute capability 10.x, else FSM_ERR_DEVICE
+ * (FSM_ERR_CUDA if the runtime cannot be queried). */
+int fsm_device_check(void);
+
+/* Bytes of device scratch fsm_index_build needs for an automaton of Q states and a
+ * vocabulary of N tokens whose byte strings total vocab_nbytes.  0 on bad sizes.
+ * Pure host arithmetic; needs no device. */
+size_t fsm_index_workspace_bytes(int32_t Q, int32_t N, int64_t vocab_nbytes);
+
+/*
+ * Vocabulary index construction (paper Section 3, Algorithms 3 and 4).
+ *
+ * For every state q in [0,Q) and every token v in [0,N) the token's bytes are
+ * walked through delta from q (Algorithm 3); the walk is abandoned at the first
+ * transition into `dead_state`, the designated absorbing state that stands for
+ * "delta undefined".  A token whose walk survives belongs to sigma(q)
+ * (Algorithm 4) and the state the walk ends in is recorded, so that the FSM
+ * state can be carried from token to token (Section 3).  Accepting states are
+ * not consulted for ordinary tokens.
+ *
+ *   dfa_trans      int32 [Q*256], row-major: dfa_trans[q*256 + b] = delta(q, b)
+ *                  (Definition 1, over the 256 byte values).  Values outside [0,Q)
+ *                  count as dead and raise FSM_FLAG_TRANS_RANGE.  The dead state's
+ *                  own row is never consulted.
+ *   accept         uint8 [Q], non-zero = state in F.
+ *   vocab_bytes    uint8 [vocab_offsets[N]], token byte strings back to back.
+ *   vocab_offsets  int32 [N+1], vocab_offsets[0] = 0, non-decreasing.  Tokens may
+ *                  have any length; a zero-length token is never allowed.
+ *   vocab_nbytes   HOST scalar equal to vocab_offsets[N] (used for bounds only).
+ *   Q, N           number of states (dead included), number of tokens.
+ *   dead_state     in [0,Q).
+ *   eos_id         token id of EOS, or -1.  EOS has no byte string: it is allowed
+ *                  exactly in accepting states and leads back to the same state.
+ *   allowed_mask   out uint32 [Q*W], W = ceil(N/32).  Bit (v & 31) of word
+ *                  q*W + (v >> 5) is 1 iff v is in sigma(q).  Every word is written;
+ *                  bits for v >= N are 0.  4-byte aligned.
+ *   next_state     out [Q*N] of `state_dtype`: the end state of the walk, or
+ *                  dead_state where the token is not allowed.  NULL = bitmask only.
+ *                  Aligned to its element size.
+ *   state_dtype    FSM_STATE_I32, or FSM_STATE_U16 (requires Q <= 65535).
+ *   workspace      device scratch, 256-byte aligned, at least
+ *                  fsm_index_workspace_bytes(Q, N, vocab_nbytes) bytes.  Contents on
+ *                  entry are irrelevant; concurrent calls need separate workspaces.
+ *   status_word    device int32 or NULL.
+ *
+ * fsm_index_build_rows builds only rows q_begin <= q < q_end, written to
+ * allowed_mask[(q - q_begin)*W ..] and next_state[(q - q_begin)*N ..]; it is the
+ * unit of work when the states are sharded over several GPUs.
+ */
+int fsm_index_build(const int32_t* dfa_trans, const uint8_t* accept,
+                    const uint8_t* vocab_bytes, const int32_t* vocab_offsets,
+                    int64_t vocab_nbytes, int32_t Q, int32_t N, int32_t dead_state,
+                    int32_t eos_id, uint32_t* allowed_mask, void* next_state,
+                    int32_t state_dtype, void* workspace, size_t workspace_bytes,
+                    int32_t* status_word, void* cuda_stream);
+
+int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* accept,
+                         const uint8_t* vocab_bytes, const int32_t* vocab_offsets,
+                         int64_t vocab_nbytes, int32_t Q, int32_t N, int32_t dead_state,
+                         int32_t eos_id, int32_t q_begin, int32_t q_end,
+                         uint32_t* allowed_mask, void* next_state, int32_t state_dtype,
+                         void* workspace, size_t workspace_bytes, int32_t* status_word,
+                         void* cuda_stream);
+
+/*
+ * One step of guided greedy decoding for a batch (paper Algorithm 2, with the
+ * greedy selection rule of Section 2.1 in place of the categorical draw).
+ *
+ * For every row i with finished[i] == 0, with q = states[i]:
+ *   mask    logits_out[i][v] = logits_in[i][v] (bit for bit) if v is in sigma(q),
+ *           else -inf  (the boolean mask m of Section 2.2 applied to the logits);
+ *   select  tok = the allowed token with the largest logit, compared as IEEE
+ *           floats (so -0.0 == +0.0); ties go to the lowest token id; NaN logits
+ *           are outside the contract;
+ *   advance if no token is allowed: finished[i] = 2, tokens_out[i] = -1;
+ *           else if tok == eos_id:  finished[i] = 1, tokens_out[i] = tok;
+ *           else tokens_out[i] = tok and states[i] = next_state[q*N + tok].
+ * Rows with finished[i] != 0 are left untouched (their logits_out row is not
+ * written) and report tokens_out[i] = -1.
+ *
+ *   logits_in    [B*row_stride] of `logits_dtype`, 16-byte aligned; row i starts
+ *                at element i*row_stride.  row_stride >= N and row_stride*sizeof
+ *                (element) a multiple of 16.
+ *   logits_out   same layout; may equal logits_in (in place) or be NULL (select and
+ *                advance only).  Partial overlap is not allowed.
+ *   states       int32 [B], in/out.  A value outside [0,Q) finishes the row as stuck
+ *                and raises FSM_FLAG_STATE_RANGE.
+ *   finished     uint8 [B], in/out: 0 live, 1 finished by EOS, 2 stuck.
+ *   tokens_out   int32 [B], out.
+ *   allowed_mask, next_state, state_dtype, Q, N, dead_state, eos_id
+ *                the index as fsm_index_build wrote it (all Q rows).
+ *   B            batch rows, >= 0 (0 is a no-op).
+ */
+int guided_mask_step(const void* logits_in, void* logits_out, int32_t logits_dtype,
+                     int64_t row_stride, int32_t* states, uint8_t* finished,
+                     int32_t* tokens_out, const uint32_t* allowed_mask,
+                     const void* next_state, int32_t state_dtype, int32_t Q, int32_t N,
+                     int32_t B, int32_t dead_state, int32_t eos_id, int32_t* status_word,
+                     void* cuda_stream);
+
+/*
+ * Tuning and test hooks (no counterpart in the paper).  Sets a process-wide knob
+ * and returns the previous value, or FSM_ERR_RANGE for an unknown key.  Not
+ * thread-safe against concurrent library calls.
+ */
+#define FSM_DEBUG_WEAK_HASH 1       /* non-zero: hash every transition column alike, so that
+                                       byte-class verification fails and the exact
+                                       uncompressed path is exercised */
+#define FSM_TUNE_MASK_CLUSTER 2     /* CTAs per logits row in guided_mask_step: 1,2,4,8; 0 = auto */
+#define FSM_TUNE_WALK_CTAS 3        /* CTAs of the walk kernel; 0 = one per SM */
+#define FSM_TUNE_SMEM_TABLE_BYTES 4 /* cap on the shared-memory table tile; 0 = device maximum */
+int fsm_debug_set(int32_t key, int32_t value);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FSMGUIDE_H */

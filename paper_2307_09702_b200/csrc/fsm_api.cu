@@ -1,0 +1,74 @@
+// Status strings, device query and process-wide knobs of the fsmguide C ABI.
+#include "fsm_common.cuh"
+
+namespace fsm {
+
+Tunables& tunables() {
+    static Tunables t;
+    return t;
+}
+
+const DeviceInfo& device_info() {
+    constexpr int kMaxDevices = 64;
+    static DeviceInfo cache[kMaxDevices] = {};
+    static DeviceInfo bad = {0, 0, 0, 0};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        return bad;
+    }
+    DeviceInfo& d = cache[dev];
+    if (!d.ok) {
+        int major = 0, sms = 0, smem = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) !=
+                cudaSuccess) {
+            (void)cudaGetLastError();
+            return bad;
+        }
+        d.cc_major = major;
+        d.sm_count = sms;
+        d.smem_optin = smem;
+        d.ok = 1;
+    }
+    return d;
+}
+
+}  // namespace fsm
+
+extern "C" const char* fsm_status_string(int status) {
+    switch (status) {
+        case FSM_OK: return "FSM_OK";
+        case FSM_ERR_NULL: return "FSM_ERR_NULL: a required pointer is NULL";
+        case FSM_ERR_SHAPE: return "FSM_ERR_SHAPE: a size is non-positive or inconsistent";
+        case FSM_ERR_ALIGN: return "FSM_ERR_ALIGN: a pointer or stride is misaligned";
+        case FSM_ERR_DTYPE: return "FSM_ERR_DTYPE: unknown dtype, or u16 states with Q > 65535";
+        case FSM_ERR_WORKSPACE: return "FSM_ERR_WORKSPACE: workspace missing or too small";
+        case FSM_ERR_RANGE: return "FSM_ERR_RANGE: dead_state, eos_id, row range or key out of range";
+        case FSM_ERR_CUDA: return "FSM_ERR_CUDA: a CUDA runtime call failed";
+        case FSM_ERR_DEVICE: return "FSM_ERR_DEVICE: current device is not compute capability 10.x";
+        default: return "FSM_ERR_UNKNOWN";
+    }
+}
+
+extern "C" int fsm_device_check(void) {
+    const fsm::DeviceInfo& d = fsm::device_info();
+    if (!d.ok) return FSM_ERR_CUDA;
+    return d.cc_major == 10 ? FSM_OK : FSM_ERR_DEVICE;
+}
+
+extern "C" int fsm_debug_set(int32_t key, int32_t value) {
+    fsm::Tunables& t = fsm::tunables();
+    int* slot = nullptr;
+    switch (key) {
+        case FSM_DEBUG_WEAK_HASH: slot = &t.weak_hash; break;
+        case FSM_TUNE_MASK_CLUSTER: slot = &t.mask_cluster; break;
+        case FSM_TUNE_WALK_CTAS: slot = &t.walk_ctas; break;
+        case FSM_TUNE_SMEM_TABLE_BYTES: slot = &t.smem_table_cap; break;
+        default: return FSM_ERR_RANGE;
+    }
+    int old = *slot;
+    *slot = value;
+    return old;
+}

@@ -1,0 +1,484 @@
+// Vocabulary index construction (paper Section 3, Algorithms 3 and 4) for sm_100a.
+//
+// Four launches on the caller's stream, no host synchronisation:
+//   1. hash_columns    one pass over delta: a 64-bit hash of each of the 256 byte columns
+//   2. derive_classes  bytes with equal column hashes share a byte class
+//   3. prepare_inputs  (a) class-compressed table [Q x Cs] with exact verification that
+//                      every byte's column equals its class representative's column,
+//                      (b) token bytes translated to class ids in 16-byte records
+//   4. walk            every (state, token) pair: one warp owns 32 consecutive tokens
+//                      (lane = token) and a run of 32 states; the table (or the tile of
+//                      start states) is staged in shared memory by bulk async copy; a
+//                      warp ballot gives the bitmask word, the end states go out as one
+//                      coalesced store per state.
+// If verification in 3(a) fails (a 64-bit hash collision) the walk reads the
+// uncompressed table instead, so the result is exact in every case.
+#include "fsm_common.cuh"
+
+namespace fsm {
+namespace {
+
+constexpr int kHashBlocks = 128;
+constexpr int kMaxCs = 264;            // 256 classes + the null class, rounded up to 8
+constexpr int kWalkThreads = 1024;
+constexpr int kWalkWarps = kWalkThreads / 32;
+constexpr int kChunk = 32;             // states per warp task
+constexpr int kInlineBytes = 16;       // token bytes kept in registers
+constexpr uint32_t kBulkChunk = 32768; // bytes per bulk copy instruction
+
+struct IndexMeta {
+    int32_t C;        // number of byte classes (the null class has id C)
+    int32_t Cs;       // row stride of the compressed table, entries
+    int32_t any_bad;  // set when a byte's column differs from its representative's
+    int32_t pad;
+};
+
+struct Workspace {
+    IndexMeta* meta;
+    uint8_t* cls;        // [256] byte -> class
+    uint8_t* class_rep;  // [256] class -> representative byte
+    uint64_t* partial;   // [kHashBlocks][256]
+    void* table;         // [Q][kMaxCs] of TabT (row stride Cs once known)
+    uint4* tok_cls;      // [G*32] first 16 class ids of each token
+    uint8_t* tok_len;    // [G*32] min(length, 17)
+    size_t bytes;
+};
+
+size_t table_elem_bytes(int32_t Q) { return Q <= 65535 ? 2 : 4; }
+
+Workspace carve(void* base, int32_t Q, int32_t N) {
+    Workspace w;
+    uint8_t* p = static_cast<uint8_t*>(base);
+    size_t off = 0;
+    auto take = [&](size_t n) {
+        uint8_t* r = p ? p + off : nullptr;
+        off += align_up(n, 256);
+        return r;
+    };
+    const size_t G = (static_cast<size_t>(N) + 31) / 32;
+    w.meta = reinterpret_cast<IndexMeta*>(take(sizeof(IndexMeta)));
+    w.cls = take(256);
+    w.class_rep = take(256);
+    w.partial = reinterpret_cast<uint64_t*>(take(sizeof(uint64_t) * kHashBlocks * 256));
+    w.table = take(static_cast<size_t>(Q) * kMaxCs * table_elem_bytes(Q));
+    w.tok_cls = reinterpret_cast<uint4*>(take(G * 32 * sizeof(uint4)));
+    w.tok_len = take(G * 32);
+    w.bytes = off;
+    return w;
+}
+
+__device__ __forceinline__ uint64_t mix64(uint64_t x) {
+    x += 0x9E3779B97F4A7C15ull;
+    x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+    x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+    return x ^ (x >> 31);
+}
+
+__device__ __forceinline__ uint32_t clamp_state(int32_t v, int32_t Q, int32_t dead) {
+    return (static_cast<uint32_t>(v) >= static_cast<uint32_t>(Q)) ? dead : v;
+}
+
+// ---------------------------------------------------------------------------- 1
+// Thread b owns byte column b; a block strides over rows.  The per-column hash is
+// a wrap-around sum of mixed (row, value) pairs, so equal columns hash alike and
+// partial sums from different blocks simply add.
+__global__ void __launch_bounds__(256) hash_columns(const int32_t* __restrict__ trans, int32_t Q,
+                                                   int32_t dead, uint64_t* __restrict__ partial,
+                                                   int weak, int32_t* status) {
+    const int b = threadIdx.x;
+    uint64_t h = 0;
+    bool bad = false;
+    for (int q = blockIdx.x; q < Q; q += gridDim.x) {
+        if (q == dead) continue;
+        int32_t v = trans[static_cast<size_t>(q) * 256 + b];
+        bad |= static_cast<uint32_t>(v) >= static_cast<uint32_t>(Q);
+        h += mix64((static_cast<uint64_t>(q) << 32) | static_cast<uint32_t>(v));
+    }
+    partial[blockIdx.x * 256 + b] = weak ? 0 : h;
+    if (__syncthreads_or(bad) && threadIdx.x == 0) raise_flag(status, FSM_FLAG_TRANS_RANGE);
+}
+
+// ---------------------------------------------------------------------------- 2
+__global__ void __launch_bounds__(256) derive_classes(const uint64_t* __restrict__ partial,
+                                                     int nblocks, IndexMeta* meta,
+                                                     uint8_t* cls, uint8_t* class_rep) {
+    __shared__ uint64_t h[256];
+    __shared__ int rep[256];
+    const int b = threadIdx.x;
+    uint64_t sum = 0;
+    for (int k = 0; k < nblocks; ++k) sum += partial[k * 256 + b];
+    h[b] = sum;
+    __syncthreads();
+    int r = b;
+    for (int k = 0; k < b; ++k)
+        if (h[k] == sum) {
+            r = k;
+            break;
+        }
+    rep[b] = r;
+    __syncthreads();
+    int id = 0;  // rank of my representative among the representatives
+    for (int k = 0; k < r; ++k) id += (rep[k] == k);
+    cls[b] = static_cast<uint8_t>(id);
+    if (r == b) class_rep[id] = static_cast<uint8_t>(b);
+    int is_rep = (r == b);
+    int C = __syncthreads_count(is_rep);
+    if (b == 0) {
+        meta->C = C;
+        meta->Cs = (C + 1 + 7) & ~7;
+        // 256 distinct columns leave no byte value for the null class: such a table
+        // is walked uncompressed.
+        meta->any_bad = (C > 255) ? 1 : 0;
+        meta->pad = 0;
+    }
+}
+
+// ---------------------------------------------------------------------------- 3
+// Blocks [0, row_blocks) compress and verify table rows; the remaining blocks
+// translate tokens.  Column C of the compressed table (the null class) and the
+// padding columns lead to the dead state, as does the whole row of the dead state.
+template <typename TabT>
+__global__ void __launch_bounds__(256)
+prepare_inputs(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab_bytes,
+               const int32_t* __restrict__ vocab_offsets, int64_t vocab_nbytes, int32_t Q,
+               int32_t N, int32_t dead, int32_t eos_id, int row_blocks, IndexMeta* meta,
+               const uint8_t* __restrict__ cls, const uint8_t* __restrict__ class_rep,
+               TabT* __restrict__ table, uint4* __restrict__ tok_cls,
+               uint8_t* __restrict__ tok_len, int32_t* status) {
+    const int C = meta->C, Cs = meta->Cs;
+    if (static_cast<int>(blockIdx.x) < row_blocks) {
+        __shared__ int32_t row[256];
+        __shared__ uint8_t s_cls[256], s_rep[256];
+        s_cls[threadIdx.x] = cls[threadIdx.x];
+        s_rep[threadIdx.x] = class_rep[threadIdx.x];
+        bool bad = false;
+        for (int q = blockIdx.x; q < Q; q += row_blocks) {
+            __syncthreads();
+            row[threadIdx.x] = clamp_state(trans[static_cast<size_t>(q) * 256 + threadIdx.x], Q, dead);
+            __syncthreads();
+            if (q != dead) bad |= row[threadIdx.x] != row[s_rep[s_cls[threadIdx.x]]];
+            for (int c = threadIdx.x; c < Cs; c += 256) {
+                int32_t v = (q == dead || c >= C) ? dead : row[s_rep[c]];
+                table[static_cast<size_t>(q) * Cs + c] = static_cast<TabT>(v);
+            }
+        }
+        if (__syncthreads_or(bad) && threadIdx.x == 0) {
+            atomicExch(&meta->any_bad, 1);
+            raise_flag(status, FSM_FLAG_CLASS_SPLIT);
+        }
+    } else {
+        const int64_t slots = (static_cast<int64_t>(N) + 31) / 32 * 32;
+        const int64_t v = static_cast<int64_t>(blockIdx.x - row_blocks) * 256 + threadIdx.x;
+        if (v >= slots) return;
+        uint32_t w[4] = {static_cast<uint32_t>(C), 0, 0, 0};  // an empty token reads the null class
+        int len = 0;
+        if (v < N && v != eos_id) {
+            const int64_t o0 = vocab_offsets[v], o1 = vocab_offsets[v + 1];
+            if (o0 < 0 || o1 < o0 || o1 > vocab_nbytes) {
+                raise_flag(status, FSM_FLAG_OFFSETS);
+            } else {
+                len = static_cast<int>(min(o1 - o0, static_cast<int64_t>(kInlineBytes + 1)));
+                const int n = min(len, kInlineBytes);
+                if (n > 0) w[0] = 0;
+                for (int i = 0; i < n; ++i)
+                    w[i >> 2] |= static_cast<uint32_t>(cls[vocab_bytes[o0 + i]]) << ((i & 3) * 8);
+            }
+        }
+        tok_cls[v] = make_uint4(w[0], w[1], w[2], w[3]);
+        tok_len[v] = static_cast<uint8_t>(len);
+    }
+}
+
+// ---------------------------------------------------------------------------- 4
+struct WalkParams {
+    const void* table;
+    const uint4* tok_cls;
+    const uint8_t* tok_len;
+    const IndexMeta* meta;
+    const int32_t* trans;
+    const uint8_t* accept;
+    const uint8_t* vocab_bytes;
+    const int32_t* vocab_offsets;
+    int64_t vocab_nbytes;
+    int32_t Q, N, G, dead, eos_id, q_begin, q_end;
+    uint32_t smem_cap;  // bytes of dynamic shared memory available for the table tile
+    uint32_t* mask;
+    void* next;
+    int32_t* status;
+};
+
+__device__ __forceinline__ uint32_t tok_byte(const uint4& t, int i) {
+    const uint32_t w = (i >> 2) == 0 ? t.x : (i >> 2) == 1 ? t.y : (i >> 2) == 2 ? t.z : t.w;
+    return (w >> ((i & 3) * 8)) & 0xFFu;
+}
+
+// Walks bytes [from, len) of token v through the uncompressed table.
+__device__ __noinline__ uint32_t raw_walk(const WalkParams& p, uint32_t s, int64_t o0, int64_t o1,
+                                          int from) {
+    for (int64_t i = o0 + from; i < o1 && s != static_cast<uint32_t>(p.dead); ++i)
+        s = clamp_state(p.trans[static_cast<size_t>(s) * 256 + p.vocab_bytes[i]], p.Q, p.dead);
+    return s;
+}
+
+template <typename OutT, bool HAS_OUT>
+__device__ __forceinline__ void emit(const WalkParams& p, int q, int g, int v, int lane, uint32_t s) {
+    const size_t r = static_cast<size_t>(q - p.q_begin);
+    if (HAS_OUT && v < p.N) static_cast<OutT*>(p.next)[r * p.N + v] = static_cast<OutT>(s);
+    const uint32_t word = __ballot_sync(kFullWarp, s != static_cast<uint32_t>(p.dead));
+    if (lane == 0) p.mask[r * p.G + g] = word;
+}
+
+// One warp task: tokens 32g .. 32g+31 (lane = token) from states q0 .. q0+nq-1.
+// `first` points at row q0 of the shared-memory tile; `tab` is the table used for
+// the second and later bytes (the same tile when FULL, else global memory).
+template <typename TabT, typename OutT, bool HAS_OUT, bool FULL>
+__device__ __forceinline__ void walk_task(const WalkParams& p, const TabT* __restrict__ first,
+                                          const TabT* __restrict__ tab, int Cs, int q0, int nq,
+                                          int g, int lane) {
+    const int v = g * 32 + lane;
+    const uint4 tk = p.tok_cls[v];
+    const int len = p.tok_len[v];
+    const uint32_t dead = p.dead;
+    const bool multi = len > 1;
+    const bool has_eos = (p.eos_id >= 0) && ((p.eos_id >> 5) == g);
+    const bool eos_lane = (v == p.eos_id);
+    const TabT* f = first + (tk.x & 0xFFu);
+    for (int j = 0; j < nq; ++j) {
+        const int q = q0 + j;
+        uint32_t s = f[static_cast<size_t>(j) * Cs];
+        bool cont = multi && (s != dead);
+        if (__any_sync(kFullWarp, cont)) {
+#pragma unroll
+            for (int i = 1; i < kInlineBytes; ++i) {
+                if (cont) {
+                    const uint32_t c = tok_byte(tk, i);
+                    if (FULL)
+                        s = tab[s * static_cast<uint32_t>(Cs) + c];
+                    else
+                        s = __ldg(tab + static_cast<size_t>(s) * Cs + c);
+                    cont = (s != dead) && (i + 1 < len);
+                }
+                if (!__any_sync(kFullWarp, cont)) break;
+            }
+            if (cont) {  // longer than the inline record: finish on the raw bytes
+                const int64_t o0 = p.vocab_offsets[v], o1 = p.vocab_offsets[v + 1];
+                s = raw_walk(p, s, o0, o1, kInlineBytes);
+            }
+        }
+        if (has_eos && eos_lane) s = (q != p.dead && p.accept[q]) ? q : dead;
+        emit<OutT, HAS_OUT>(p, q, g, v, lane, s);
+    }
+}
+
+// Same task on the uncompressed table (exact fallback after a class split).
+template <typename OutT, bool HAS_OUT>
+__device__ __noinline__ void walk_task_raw(const WalkParams& p, int q0, int nq, int g, int lane) {
+    const int v = g * 32 + lane;
+    int64_t o0 = 0, o1 = 0;
+    if (v < p.N && v != p.eos_id) {
+        o0 = p.vocab_offsets[v];
+        o1 = p.vocab_offsets[v + 1];
+        if (o0 < 0 || o1 < o0 || o1 > p.vocab_nbytes) o0 = o1 = 0;
+    }
+    for (int j = 0; j < nq; ++j) {
+        const int q = q0 + j;
+        uint32_t s = p.dead;
+        if (o1 > o0 && q != p.dead) s = raw_walk(p, q, o0, o1, 0);
+        if (v == p.eos_id) s = (q != p.dead && p.accept[q]) ? q : p.dead;
+        emit<OutT, HAS_OUT>(p, q, g, v, lane, s);
+    }
+}
+
+template <typename TabT, typename OutT, bool HAS_OUT>
+__global__ void __launch_bounds__(kWalkThreads, 1) walk(const WalkParams p) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    __shared__ uint64_t bar;
+    TabT* tile = reinterpret_cast<TabT*>(smem_raw);
+    const TabT* gtab = static_cast<const TabT*>(p.table);
+    const int Cs = p.meta->Cs;
+    const bool raw = p.meta->any_bad != 0;
+    const uint32_t row_bytes = Cs * sizeof(TabT);
+    const int nrows = p.q_end - p.q_begin;
+    const bool full = static_cast<uint64_t>(p.Q) * row_bytes <= p.smem_cap;
+    const int cap_rows = max(kChunk, static_cast<int>(p.smem_cap / row_bytes) / kChunk * kChunk);
+    const int ntiles = full ? 1 : (nrows + cap_rows - 1) / cap_rows;
+    const int lane = threadIdx.x & 31;
+    const int64_t wg = static_cast<int64_t>(blockIdx.x) * kWalkWarps + (threadIdx.x >> 5);
+    const int64_t TW = static_cast<int64_t>(gridDim.x) * kWalkWarps;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    uint32_t parity = 0;
+    for (int ti = 0; ti < ntiles; ++ti) {
+        const int t_q0 = full ? 0 : p.q_begin + ti * cap_rows;          // first staged row
+        const int t_rows = full ? p.Q : min(cap_rows, p.q_end - t_q0);  // staged rows
+        const int w_q0 = full ? p.q_begin : t_q0;                       // first start state
+        const int w_rows = full ? nrows : t_rows;
+        if (!raw) {
+            if (ti > 0) __syncthreads();  // every warp is done with the previous tile
+            if (threadIdx.x == 0) {
+                const uint32_t bytes = static_cast<uint32_t>(t_rows) * row_bytes;
+                const uint8_t* src =
+                    reinterpret_cast<const uint8_t*>(gtab) + static_cast<size_t>(t_q0) * row_bytes;
+                mbar_expect_tx(&bar, bytes);
+                for (uint32_t o = 0; o < bytes; o += kBulkChunk)
+                    bulk_copy_g2s(smem_raw + o, src + o, min(kBulkChunk, bytes - o), &bar);
+            }
+            bool ok = mbar_wait_bounded(&bar, parity);
+            if (!ok) ok = mbar_wait_bounded(&bar, parity);  // drain before giving up
+            parity ^= 1;
+            if (!__syncthreads_and(ok)) {
+                if (threadIdx.x == 0) raise_flag(p.status, FSM_FLAG_WAIT_TIMEOUT);
+                return;
+            }
+        }
+        const int nchunks = (w_rows + kChunk - 1) / kChunk;
+        const int64_t ntasks = static_cast<int64_t>(nchunks) * p.G;
+        for (int64_t t = wg; t < ntasks; t += TW) {
+            const int chunk = static_cast<int>(t / p.G);
+            const int g = static_cast<int>(t - static_cast<int64_t>(chunk) * p.G);
+            const int q0 = w_q0 + chunk * kChunk;
+            const int nq = min(kChunk, w_q0 + w_rows - q0);
+            if (raw) {
+                walk_task_raw<OutT, HAS_OUT>(p, q0, nq, g, lane);
+            } else {
+                const TabT* first = tile + static_cast<size_t>(q0 - t_q0) * Cs;
+                if (full)
+                    walk_task<TabT, OutT, HAS_OUT, true>(p, first, tile, Cs, q0, nq, g, lane);
+                else
+                    walk_task<TabT, OutT, HAS_OUT, false>(p, first, gtab, Cs, q0, nq, g, lane);
+            }
+        }
+    }
+}
+
+template <typename TabT, typename OutT, bool HAS_OUT>
+cudaError_t launch_walk(const WalkParams& p, int grid, cudaStream_t stream) {
+    auto kernel = walk<TabT, OutT, HAS_OUT>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(p.smem_cap));
+    if (e != cudaSuccess) return e;
+    kernel<<<grid, kWalkThreads, p.smem_cap, stream>>>(p);
+    return cudaGetLastError();
+}
+
+template <typename TabT>
+cudaError_t launch_walk_for(const WalkParams& p, int grid, int32_t state_dtype, bool has_out,
+                            cudaStream_t stream) {
+    if (!has_out) return launch_walk<TabT, int32_t, false>(p, grid, stream);
+    if (state_dtype == FSM_STATE_U16) return launch_walk<TabT, uint16_t, true>(p, grid, stream);
+    return launch_walk<TabT, int32_t, true>(p, grid, stream);
+}
+
+}  // namespace
+}  // namespace fsm
+
+extern "C" size_t fsm_index_workspace_bytes(int32_t Q, int32_t N, int64_t vocab_nbytes) {
+    if (Q <= 0 || N <= 0 || vocab_nbytes < 0) return 0;
+    return fsm::carve(nullptr, Q, N).bytes;
+}
+
+extern "C" int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* accept,
+                                    const uint8_t* vocab_bytes, const int32_t* vocab_offsets,
+                                    int64_t vocab_nbytes, int32_t Q, int32_t N,
+                                    int32_t dead_state, int32_t eos_id, int32_t q_begin,
+                                    int32_t q_end, uint32_t* allowed_mask, void* next_state,
+                                    int32_t state_dtype, void* workspace, size_t workspace_bytes,
+                                    int32_t* status_word, void* cuda_stream) {
+    using namespace fsm;
+    if (Q <= 0 || N <= 0 || vocab_nbytes < 0 || N > 0x7FFFFFE0) return FSM_ERR_SHAPE;
+    if (!dfa_trans || !accept || !vocab_offsets || !allowed_mask) return FSM_ERR_NULL;
+    if (!vocab_bytes && vocab_nbytes > 0) return FSM_ERR_NULL;
+    if (state_dtype != FSM_STATE_I32 && state_dtype != FSM_STATE_U16) return FSM_ERR_DTYPE;
+    if (state_dtype == FSM_STATE_U16 && Q > 65535) return FSM_ERR_DTYPE;
+    if (dead_state < 0 || dead_state >= Q) return FSM_ERR_RANGE;
+    if (eos_id < -1 || eos_id >= N) return FSM_ERR_RANGE;
+    if (q_begin < 0 || q_end > Q || q_begin > q_end) return FSM_ERR_RANGE;
+    auto misaligned = [](const void* p, size_t a) { return reinterpret_cast<uintptr_t>(p) % a != 0; };
+    if (misaligned(dfa_trans, 4) || misaligned(vocab_offsets, 4) || misaligned(allowed_mask, 4) ||
+        misaligned(status_word, 4))
+        return FSM_ERR_ALIGN;
+    if (next_state && misaligned(next_state, state_dtype == FSM_STATE_U16 ? 2 : 4))
+        return FSM_ERR_ALIGN;
+    const size_t need = fsm_index_workspace_bytes(Q, N, vocab_nbytes);
+    if (!workspace || workspace_bytes < need) return FSM_ERR_WORKSPACE;
+    if (misaligned(workspace, 256)) return FSM_ERR_ALIGN;
+    if (q_begin == q_end) return FSM_OK;
+
+    const DeviceInfo& dev = device_info();
+    if (!dev.ok) return FSM_ERR_CUDA;
+    if (dev.cc_major != 10) return FSM_ERR_DEVICE;
+    const Tunables& tune = tunables();
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    Workspace ws = carve(workspace, Q, N);
+    const bool wide = Q > 65535;
+
+    const int hash_blocks = Q < kHashBlocks ? Q : kHashBlocks;
+    hash_columns<<<hash_blocks, 256, 0, stream>>>(dfa_trans, Q, dead_state, ws.partial,
+                                                  tune.weak_hash, status_word);
+    derive_classes<<<1, 256, 0, stream>>>(ws.partial, hash_blocks, ws.meta, ws.cls, ws.class_rep);
+    const int G = (N + 31) / 32;
+    const int row_blocks = Q < 2 * dev.sm_count ? Q : 2 * dev.sm_count;
+    const int tok_blocks = (G * 32 + 255) / 256;
+    if (wide)
+        prepare_inputs<int32_t><<<row_blocks + tok_blocks, 256, 0, stream>>>(
+            dfa_trans, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
+            row_blocks, ws.meta, ws.cls, ws.class_rep, static_cast<int32_t*>(ws.table),
+            ws.tok_cls, ws.tok_len, status_word);
+    else
+        prepare_inputs<uint16_t><<<row_blocks + tok_blocks, 256, 0, stream>>>(
+            dfa_trans, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
+            row_blocks, ws.meta, ws.cls, ws.class_rep, static_cast<uint16_t*>(ws.table),
+            ws.tok_cls, ws.tok_len, status_word);
+    if (cudaGetLastError() != cudaSuccess) return FSM_ERR_CUDA;
+
+    WalkParams p;
+    p.table = ws.table;
+    p.tok_cls = ws.tok_cls;
+    p.tok_len = ws.tok_len;
+    p.meta = ws.meta;
+    p.trans = dfa_trans;
+    p.accept = accept;
+    p.vocab_bytes = vocab_bytes;
+    p.vocab_offsets = vocab_offsets;
+    p.vocab_nbytes = vocab_nbytes;
+    p.Q = Q;
+    p.N = N;
+    p.G = G;
+    p.dead = dead_state;
+    p.eos_id = eos_id;
+    p.q_begin = q_begin;
+    p.q_end = q_end;
+    p.mask = allowed_mask;
+    p.next = next_state;
+    p.status = status_word;
+    int cap = dev.smem_optin - 1024;  // static shared memory and alignment slack
+    if (tune.smem_table_cap > 0 && tune.smem_table_cap < cap) cap = tune.smem_table_cap;
+    const int min_cap = kChunk * kMaxCs * 4;
+    if (cap < min_cap) cap = min_cap;
+    p.smem_cap = static_cast<uint32_t>(cap) / 128 * 128;
+
+    const int64_t tasks = static_cast<int64_t>((q_end - q_begin + kChunk - 1) / kChunk) * G;
+    int64_t grid = (tasks + kWalkWarps - 1) / kWalkWarps;
+    if (grid > dev.sm_count) grid = dev.sm_count;
+    if (tune.walk_ctas > 0) grid = tune.walk_ctas;
+    cudaError_t e = wide ? launch_walk_for<int32_t>(p, static_cast<int>(grid), state_dtype,
+                                                   next_state != nullptr, stream)
+                         : launch_walk_for<uint16_t>(p, static_cast<int>(grid), state_dtype,
+                                                    next_state != nullptr, stream);
+    return e == cudaSuccess ? FSM_OK : FSM_ERR_CUDA;
+}
+
+extern "C" int fsm_index_build(const int32_t* dfa_trans, const uint8_t* accept,
+                               const uint8_t* vocab_bytes, const int32_t* vocab_offsets,
+                               int64_t vocab_nbytes, int32_t Q, int32_t N, int32_t dead_state,
+                               int32_t eos_id, uint32_t* allowed_mask, void* next_state,
+                               int32_t state_dtype, void* workspace, size_t workspace_bytes,
+                               int32_t* status_word, void* cuda_stream) {
+    return fsm_index_build_rows(dfa_trans, accept, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N,
+                                dead_state, eos_id, 0, Q, allowed_mask, next_state, state_dtype,
+                                workspace, workspace_bytes, status_word, cuda_stream);
+}

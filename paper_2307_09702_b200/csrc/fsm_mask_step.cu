@@ -1,0 +1,298 @@
+// Masked greedy decode step (paper Algorithm 2 with argmax selection) for sm_100a.
+//
+// One thread-block cluster of `k` CTAs owns one logits row.  Each thread streams
+// 32-byte vectors of the row: it first reads the vector's bits of the allowed-token
+// bitmask row sigma(state) (L2 resident), loads the logits only when at least one
+// bit is set (a vector with no allowed token becomes -inf whatever it held), writes
+// the masked vector and keeps a running (value, lowest id) maximum over the allowed
+// entries.  The maxima are reduced by warp shuffles, through shared memory, and
+// across the cluster through distributed shared memory; the cluster's first CTA
+// then looks up the next state and updates states / finished / tokens_out.
+#include <cooperative_groups.h>
+
+#include "fsm_common.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace fsm {
+namespace {
+
+constexpr int kStepThreads = 256;
+constexpr int kStepWarps = kStepThreads / 32;
+constexpr int kNone = 0x7FFFFFFF;
+
+struct StepParams {
+    const void* in;
+    void* out;
+    int64_t row_stride;
+    int32_t* states;
+    uint8_t* finished;
+    int32_t* tokens;
+    const uint32_t* mask;
+    const void* next;
+    int32_t state_u16;
+    int32_t Q, N, W, B, dead, eos_id, k;
+    int32_t* status;
+};
+
+struct Best {
+    float val;
+    int idx;
+};
+
+// `b` replaces `a` when it is the better candidate: larger value, or equal value
+// and lower id; kNone marks "no allowed token seen".
+__device__ __forceinline__ Best better(Best a, Best b) {
+    const bool take = (b.idx != kNone) &&
+                      (a.idx == kNone || b.val > a.val || (b.val == a.val && b.idx < a.idx));
+    return take ? b : a;
+}
+
+template <typename T> struct Elem;
+template <> struct Elem<uint32_t> {  // fp32 bit patterns
+    static constexpr int kPerWord = 1;
+    static constexpr uint32_t kNegInfWord = 0xFF800000u;
+    __device__ static float get(uint32_t w, int) { return __uint_as_float(w); }
+    __device__ static uint32_t select(uint32_t w, uint32_t bits) { return (bits & 1u) ? w : kNegInfWord; }
+};
+template <> struct Elem<uint16_t> {  // bf16 bit patterns
+    static constexpr int kPerWord = 2;
+    static constexpr uint32_t kNegInfWord = 0xFF80FF80u;
+    __device__ static float get(uint32_t w, int j) { return __uint_as_float(j ? (w & 0xFFFF0000u) : (w << 16)); }
+    __device__ static uint32_t select(uint32_t w, uint32_t bits) {
+        const uint32_t keep = ((bits & 1u) ? 0x0000FFFFu : 0u) | ((bits & 2u) ? 0xFFFF0000u : 0u);
+        return (w & keep) | (kNegInfWord & ~keep);
+    }
+};
+
+// Processes one vector of NW 32-bit words whose first element has index e0.
+template <typename T, int NW>
+__device__ __forceinline__ void process(uint32_t (&w)[NW], uint32_t bits, int e0, Best& best) {
+    constexpr int PW = Elem<T>::kPerWord;
+#pragma unroll
+    for (int i = 0; i < NW; ++i) {
+        const uint32_t b = (bits >> (i * PW)) & ((1u << PW) - 1u);
+#pragma unroll
+        for (int j = 0; j < PW; ++j) {
+            if (b & (1u << j)) {
+                const float x = Elem<T>::get(w[i], j);
+                if (!(x <= best.val)) {  // also true for the first allowed entry (val is NaN)
+                    best.val = x;
+                    best.idx = e0 + i * PW + j;
+                }
+            }
+        }
+        w[i] = Elem<T>::select(w[i], b);
+    }
+}
+
+template <typename T, bool WRITE>
+__global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
+    cg::cluster_group cluster = cg::this_cluster();
+    __shared__ Best warp_best[kStepWarps];
+    __shared__ Best cta_best[8];  // slot r of the cluster's first CTA receives CTA r's result
+
+    const int k = p.k;
+    const int row = blockIdx.x / k;
+    const int rank = blockIdx.x - row * k;  // == cluster.block_rank() for 1-D clusters
+    // Uniform over the cluster: nobody reaches the cluster barrier for a finished row.
+    if (p.finished[row] != 0) {
+        if (rank == 0 && threadIdx.x == 0) p.tokens[row] = -1;
+        return;
+    }
+    int q = p.states[row];
+    const bool bad_state = static_cast<uint32_t>(q) >= static_cast<uint32_t>(p.Q);
+    const uint32_t* mrow = p.mask + static_cast<size_t>(bad_state ? 0 : q) * p.W;
+    const uint32_t live = bad_state ? 0u : 0xFFFFFFFFu;
+
+    constexpr int EPV = 32 / sizeof(T);   // elements per 32-byte vector
+    constexpr int EPH = 16 / sizeof(T);   // elements per 16-byte vector
+    const T* in = static_cast<const T*>(p.in) + static_cast<size_t>(row) * p.row_stride;
+    T* out = WRITE ? static_cast<T*>(p.out) + static_cast<size_t>(row) * p.row_stride : nullptr;
+    const bool wide = ((reinterpret_cast<uintptr_t>(in) | (WRITE ? reinterpret_cast<uintptr_t>(out) : 0)) & 31) == 0;
+
+    Best best{__int_as_float(0x7FC00000), kNone};
+    const int tid = rank * kStepThreads + threadIdx.x;
+    const int nthreads = k * kStepThreads;
+
+    int done = 0;  // elements covered by whole vectors
+    if (wide) {
+        const int nvec = p.N / EPV;
+        for (int vi = tid; vi < nvec; vi += nthreads) {
+            const int e0 = vi * EPV;
+            const uint32_t bits = live & (mrow[e0 >> 5] >> (e0 & 31)) & ((EPV == 32) ? 0xFFFFFFFFu : ((1u << EPV) - 1u));
+            Vec32B v;
+            if (bits != 0) {
+                v = ldg_stream_32B(in + e0);
+                process<T, 8>(v.w, bits, e0, best);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) v.w[i] = Elem<T>::kNegInfWord;
+            }
+            if (WRITE) stg_32B(out + e0, v);
+        }
+        done = nvec * EPV;
+    } else {
+        const int nvec = p.N / EPH;
+        for (int vi = tid; vi < nvec; vi += nthreads) {
+            const int e0 = vi * EPH;
+            const uint32_t bits = live & (mrow[e0 >> 5] >> (e0 & 31)) & ((1u << EPH) - 1u);
+            uint32_t w[4];
+            if (bits != 0) {
+                const uint4 v = *reinterpret_cast<const uint4*>(in + e0);
+                w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+                process<T, 4>(w, bits, e0, best);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) w[i] = Elem<T>::kNegInfWord;
+            }
+            if (WRITE) *reinterpret_cast<uint4*>(out + e0) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        done = nvec * EPH;
+    }
+    // Ragged tail (fewer elements than one vector): one element per thread of the last CTA.
+    if (rank == k - 1) {
+        const int e = done + threadIdx.x;
+        if (e < p.N) {
+            const bool allowed = (live & (mrow[e >> 5] >> (e & 31)) & 1u) != 0;
+            const T raw = in[e];
+            if (allowed) {
+                const float x = sizeof(T) == 4 ? __uint_as_float(static_cast<uint32_t>(raw))
+                                               : __uint_as_float(static_cast<uint32_t>(raw) << 16);
+                if (!(x <= best.val)) {
+                    best.val = x;
+                    best.idx = e;
+                }
+            } else if (WRITE) {
+                out[e] = static_cast<T>(sizeof(T) == 4 ? 0xFF800000u : 0xFF80u);
+            }
+            if (allowed && WRITE) out[e] = raw;
+        }
+    }
+
+    // A thread's own ids only grow, so its (val, idx) already holds the lowest id
+    // among equal values; combining needs the full ordering.
+    if (best.idx == kNone) best.val = 0.0f;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        Best o;
+        o.val = __shfl_xor_sync(kFullWarp, best.val, off);
+        o.idx = __shfl_xor_sync(kFullWarp, best.idx, off);
+        best = better(best, o);
+    }
+    if ((threadIdx.x & 31) == 0) warp_best[threadIdx.x >> 5] = best;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        Best b = warp_best[0];
+#pragma unroll
+        for (int i = 1; i < kStepWarps; ++i) b = better(b, warp_best[i]);
+        Best* dst = (k > 1) ? cluster.map_shared_rank(&cta_best[rank], 0) : &cta_best[0];
+        *dst = b;
+    }
+    if (k > 1) cluster.sync();
+    if (rank == 0 && threadIdx.x == 0) {
+        Best b = cta_best[0];
+        for (int i = 1; i < k; ++i) b = better(b, cta_best[i]);
+        if (bad_state) raise_flag(p.status, FSM_FLAG_STATE_RANGE);
+        if (b.idx == kNone) {
+            p.finished[row] = 2;
+            p.tokens[row] = -1;
+        } else if (b.idx == p.eos_id) {
+            p.finished[row] = 1;
+            p.tokens[row] = b.idx;
+        } else {
+            p.tokens[row] = b.idx;
+            const size_t at = static_cast<size_t>(q) * p.N + b.idx;
+            p.states[row] = p.state_u16 ? static_cast<int32_t>(static_cast<const uint16_t*>(p.next)[at])
+                                        : static_cast<const int32_t*>(p.next)[at];
+        }
+    }
+}
+
+template <typename T, bool WRITE>
+cudaError_t launch(const StepParams& p, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(p.B) * p.k, 1, 1);
+    cfg.blockDim = dim3(kStepThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = p.k;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, mask_step<T, WRITE>, p);
+}
+
+}  // namespace
+}  // namespace fsm
+
+extern "C" int guided_mask_step(const void* logits_in, void* logits_out, int32_t logits_dtype,
+                                int64_t row_stride, int32_t* states, uint8_t* finished,
+                                int32_t* tokens_out, const uint32_t* allowed_mask,
+                                const void* next_state, int32_t state_dtype, int32_t Q, int32_t N,
+                                int32_t B, int32_t dead_state, int32_t eos_id,
+                                int32_t* status_word, void* cuda_stream) {
+    using namespace fsm;
+    if (Q <= 0 || N <= 0 || B < 0 || row_stride < N) return FSM_ERR_SHAPE;
+    if (!logits_in || !states || !finished || !tokens_out || !allowed_mask || !next_state)
+        return FSM_ERR_NULL;
+    if (logits_dtype != FSM_LOGITS_F32 && logits_dtype != FSM_LOGITS_BF16) return FSM_ERR_DTYPE;
+    if (state_dtype != FSM_STATE_I32 && state_dtype != FSM_STATE_U16) return FSM_ERR_DTYPE;
+    if (state_dtype == FSM_STATE_U16 && Q > 65535) return FSM_ERR_DTYPE;
+    if (dead_state < 0 || dead_state >= Q || eos_id < -1 || eos_id >= N) return FSM_ERR_RANGE;
+    const size_t esize = logits_dtype == FSM_LOGITS_F32 ? 4 : 2;
+    auto misaligned = [](const void* p, size_t a) { return reinterpret_cast<uintptr_t>(p) % a != 0; };
+    if (misaligned(logits_in, 16) || misaligned(logits_out, 16) ||
+        (static_cast<uint64_t>(row_stride) * esize) % 16 != 0)
+        return FSM_ERR_ALIGN;
+    if (misaligned(states, 4) || misaligned(tokens_out, 4) || misaligned(allowed_mask, 4) ||
+        misaligned(next_state, state_dtype == FSM_STATE_U16 ? 2 : 4) || misaligned(status_word, 4))
+        return FSM_ERR_ALIGN;
+    if (static_cast<int64_t>(B) * 8 > 0x7FFFFFFF) return FSM_ERR_SHAPE;
+    if (B == 0) return FSM_OK;
+
+    const DeviceInfo& dev = device_info();
+    if (!dev.ok) return FSM_ERR_CUDA;
+    if (dev.cc_major != 10) return FSM_ERR_DEVICE;
+
+    // CTAs per row: enough CTAs to fill the device several times over, but at least
+    // a few vectors per thread.
+    int k = tunables().mask_cluster;
+    if (k != 1 && k != 2 && k != 4 && k != 8) {
+        k = 1;
+        const int64_t vectors = static_cast<int64_t>(N) * esize / 32;
+        while (k < 8 && static_cast<int64_t>(B) * k < 6LL * dev.sm_count &&
+               vectors / (2 * k * kStepThreads) >= 2)
+            k *= 2;
+    }
+
+    StepParams p;
+    p.in = logits_in;
+    p.out = logits_out;
+    p.row_stride = row_stride;
+    p.states = states;
+    p.finished = finished;
+    p.tokens = tokens_out;
+    p.mask = allowed_mask;
+    p.next = next_state;
+    p.state_u16 = state_dtype == FSM_STATE_U16;
+    p.Q = Q;
+    p.N = N;
+    p.W = (N + 31) / 32;
+    p.B = B;
+    p.dead = dead_state;
+    p.eos_id = eos_id;
+    p.k = k;
+    p.status = status_word;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e;
+    const bool write = logits_out != nullptr;
+    if (logits_dtype == FSM_LOGITS_F32)
+        e = write ? launch<uint32_t, true>(p, stream) : launch<uint32_t, false>(p, stream);
+    else
+        e = write ? launch<uint16_t, true>(p, stream) : launch<uint16_t, false>(p, stream);
+    return e == cudaSuccess ? FSM_OK : FSM_ERR_CUDA;
+}
