@@ -1,0 +1,386 @@
+#!/usr/bin/env python
+"""Benchmark of the FSM-indexed guided-generation hot path on B200.
+
+One *step* is one pass of the whole path over one batch of synthetic input:
+``fsm_index_build`` for the Llama-3-shaped workload (1,001 states x 128,256
+tokens, int32 next-state table) followed by one ``guided_mask_step`` over
+B = 256 bf16 logits rows of that vocabulary, in place.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints one JSON line.  ``value`` is (state, token) walks per second of the index
+build (Q*N per build, all ranks, divided by the build's device time inside the
+step); ``mask_step_us`` is the masked-logit step; ``ms_per_step`` is the whole
+step.  With N > 1 (torchrun) every rank runs the same-shaped workload on its own
+GPU with its own automaton seed: the path shards over independent problems and
+has no data-path collective (weak scaling).
+
+``--impl reference`` times the CPU oracle on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "index build (state,token) walks/s; masked-logit step us at B=256, N=128k"
+UNIT = "walks/s"
+B_ROWS = 256
+RING = 4
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def workload(rank: int):
+    """Workload 3 (index) + workload 5 (decode batch); rank r > 0 draws its own
+    automaton of the same shape."""
+    from fsm_inputs import make_config, random_class_dfa, start_states
+    w = make_config(5)
+    if rank > 0:
+        w.dfa, _ = random_class_dfa(w.seed + 5000 + rank, 1000, 64, 12, 0.10)
+    return w, start_states(w)
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake",
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.01)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------- CPU oracle legs
+def oracle_index_rate(w, threads, budget_s):
+    """Times the oracle's index build on a bounded sample of states."""
+    from oracle import fsm_oracle
+    d = w.dfa
+    t0 = time.perf_counter()
+    fsm_oracle.index_build(d.trans, d.accept, w.vocab_bytes, w.vocab_offsets, d.dead, w.eos_id,
+                           q_begin=0, q_end=min(16, d.Q), threads=threads)
+    per_state = max((time.perf_counter() - t0) / min(16, d.Q), 1e-6)
+    n_states = int(max(1, min(d.Q, budget_s / per_state)))
+    t0 = time.perf_counter()
+    fsm_oracle.index_build(d.trans, d.accept, w.vocab_bytes, w.vocab_offsets, d.dead, w.eos_id,
+                           q_begin=0, q_end=n_states, threads=threads)
+    dt = time.perf_counter() - t0
+    return n_states * w.N / dt, n_states, dt
+
+
+def cpu_baseline(w, starts):
+    from fsm_inputs import f32_to_bf16_bits, step_logits_numpy
+    from oracle import fsm_oracle
+    threads = len(os.sched_getaffinity(0))
+    rate, n_states, dt = oracle_index_rate(w, threads, budget_s=8.0)
+    d = w.dfa
+    mask, nxt, _ = fsm_oracle.index_build(d.trans, d.accept, w.vocab_bytes, w.vocab_offsets, d.dead,
+                                          w.eos_id, threads=threads)
+    logits = f32_to_bf16_bits(step_logits_numpy(w, 0))
+    reps, t_mask = 3, []
+    for _ in range(reps):
+        st, fin = starts.copy(), np.zeros(w.B, np.uint8)
+        t0 = time.perf_counter()
+        fsm_oracle.mask_step(logits, st, fin, mask, nxt, d.dead, w.eos_id, threads=threads)
+        t_mask.append(time.perf_counter() - t0)
+    return {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"index build of states 0..{n_states - 1} of {d.Q} x all {w.N} tokens "
+                      f"({dt:.2f} s, OpenMP over states); mask step: {reps} full B=256 steps",
+            "mask_step_us": float(np.median(t_mask) * 1e6)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w, starts = workload(0)
+    threads = len(os.sched_getaffinity(0))
+    total = max(1, args.steps + args.warmup)
+    budget = min(20.0, 150.0 / total)              # seconds of oracle work per step
+    from fsm_inputs import f32_to_bf16_bits, step_logits_numpy
+    from oracle import fsm_oracle
+    d = w.dfa
+    rate, n_states, _ = oracle_index_rate(w, threads, budget * 0.8)
+    rows = int(max(1, min(w.B, round(w.B * budget * 0.2 / 0.1))))   # ~0.1 s per full step on 8 cores
+    mask, nxt, _ = fsm_oracle.index_build(d.trans, d.accept, w.vocab_bytes, w.vocab_offsets, d.dead,
+                                          w.eos_id, threads=threads)
+    logits = f32_to_bf16_bits(step_logits_numpy(w, 0))[:rows].copy()
+    t_build, t_mask = [], []
+    for it in range(total):
+        t0 = time.perf_counter()
+        fsm_oracle.index_build(d.trans, d.accept, w.vocab_bytes, w.vocab_offsets, d.dead, w.eos_id,
+                               q_begin=0, q_end=n_states, threads=threads)
+        t1 = time.perf_counter()
+        st, fin = starts[:rows].copy(), np.zeros(rows, np.uint8)
+        fsm_oracle.mask_step(logits, st, fin, mask, nxt, d.dead, w.eos_id, threads=threads)
+        t2 = time.perf_counter()
+        if it >= args.warmup:
+            t_build.append(t1 - t0)
+            t_mask.append(t2 - t1)
+    value = n_states * w.N / float(np.mean(t_build))
+    mask_us = float(np.mean(t_mask)) * 1e6 * (w.B / rows)
+    sample = (f"per step: oracle index build of {n_states} of {d.Q} states x {w.N} tokens, and "
+              f"the oracle mask step on {rows} of {w.B} rows (scaled to {w.B})")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": float(np.mean(t_build) + np.mean(t_mask)) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32",
+        "data": "synthetic", "mask_step_us": mask_us,
+        "config": config_dict(w, args.gpus),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def config_dict(w, n_gpus):
+    return {"workload": "index build: Llama-3-shaped vocab N=128256, random DFA Q=1001 (12 live "
+                        "byte classes/state), int32 next-state + packed bitmask; then one mask "
+                        "step: B=256 bf16 logits [256x128256], in place",
+            "Q": w.Q, "N": w.N, "B": w.B, "state_dtype": "int32", "logits_dtype": "bf16",
+            "parallelism": f"independent problems x{n_gpus}, no collective",
+            "l2": f"per-step working set ~660 MB (529 MB index output written between mask steps, "
+                  f"logits ring of {RING} x 65.7 MB) exceeds the 126 MB L2; no explicit flush"}
+
+
+# --------------------------------------------------------------------------- GPU arm
+def run_ours(args):
+    import torch
+    import paper_2307_09702_b200 as fg
+    from paper_2307_09702_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if fg.fsm_device_check() != 0:
+        raise SystemExit("bench.py needs a compute-capability 10.x device")
+    dev = torch.device("cuda", local)
+    w, starts = workload(rank)
+    d = w.dfa
+    idx = fg.GuidedIndex(d.trans, d.accept, w.vocab_bytes, w.vocab_offsets, d.dead, w.eos_id,
+                         fg.FSM_STATE_I32, True, device=dev)
+    sigma = w.logits_sigma
+    g = torch.Generator(device=dev).manual_seed(w.seed)
+    ring = [(torch.randn((w.B, w.N), generator=g, device=dev) * sigma).to(torch.bfloat16)
+            for _ in range(RING)]
+    st0 = torch.from_numpy(starts).to(dev)
+    fin0 = torch.zeros(w.B, dtype=torch.uint8, device=dev)
+    st, fin = st0.clone(), fin0.clone()
+    tok = torch.zeros(w.B, dtype=torch.int32, device=dev)
+
+    def step(i, ev=None):
+        st.copy_(st0)
+        fin.copy_(fin0)
+        if ev:
+            ev[0].record()
+        idx.build()
+        if ev:
+            ev[1].record()
+        idx.step(ring[i % RING], st, fin, tok)
+        if ev:
+            ev[2].record()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    assert int(idx.status.item()) == 0, "data-fault flag raised during warm-up"
+
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    fg.fsm_debug_set(binding.FSM_PROFILE_WALK, 1)
+    sampler = ClockSampler(local)
+    sampler.start()
+    barrier()
+    t_begin.record()
+    for i in range(args.steps):
+        step(i, events[i])
+    t_end.record()
+    barrier()
+    clocks = sampler.stop()
+    fg.fsm_debug_set(binding.FSM_PROFILE_WALK, 0)
+    walk_ms = fg.fsm_profile_read()[: args.steps]
+    total_ms = t_begin.elapsed_time(t_end)
+    build_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in events]))
+    mask_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in events]))
+    walk_ms_mean = float(np.mean(walk_ms)) if walk_ms else float("nan")
+
+    # ---- end to end: host buffers in, host results out, through the same calls
+    host = {k: torch.from_numpy(np.ascontiguousarray(v)).pin_memory() for k, v in {
+        "trans": d.trans, "accept": d.accept, "vb": w.vocab_bytes, "vo": w.vocab_offsets,
+        "states": starts}.items()}
+    host_logits = ring[0].cpu().pin_memory()
+    host_fin = torch.zeros(w.B, dtype=torch.uint8).pin_memory()
+    out_tok = torch.empty(w.B, dtype=torch.int32).pin_memory()
+    out_st = torch.empty(w.B, dtype=torch.int32).pin_memory()
+    out_fin = torch.empty(w.B, dtype=torch.uint8).pin_memory()
+    dev_logits = torch.empty_like(ring[0])
+    h2d = sum(t.numel() * t.element_size() for t in host.values()) + \
+        host_logits.numel() * 2 + host_fin.numel()
+    d2h = out_tok.numel() * 4 + out_st.numel() * 4 + out_fin.numel()
+
+    def e2e_step():
+        idx.trans.copy_(host["trans"], non_blocking=True)
+        idx.accept.copy_(host["accept"], non_blocking=True)
+        idx.vocab_bytes.copy_(host["vb"], non_blocking=True)
+        idx.vocab_offsets.copy_(host["vo"], non_blocking=True)
+        dev_logits.copy_(host_logits, non_blocking=True)
+        st.copy_(host["states"], non_blocking=True)
+        fin.copy_(host_fin, non_blocking=True)
+        idx.build()
+        idx.step(dev_logits, st, fin, tok)
+        out_tok.copy_(tok, non_blocking=True)
+        out_st.copy_(st, non_blocking=True)
+        out_fin.copy_(fin, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    e2e_steps = max(3, min(args.steps, 50))
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+
+    def allmax(x):
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    total_ms, build_ms, mask_ms, walk_ms_mean, e2e_s = map(
+        allmax, (total_ms, build_ms, mask_ms, walk_ms_mean, e2e_s))
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    walks = float(w.Q) * w.N
+    hbm_gbs, peak_kind = load_peaks()
+    walk_bytes = walks * 4 + w.Q * w.W * 4                    # next-state entries + bitmask words
+    live_rows = w.B
+    mask_bytes = live_rows * w.N * 2 * 2 + live_rows * w.W * 4
+    achieved = walk_bytes / (walk_ms_mean * 1e-3) / 1e9
+    mask_achieved = mask_bytes / (mask_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": walks * world / (build_ms * 1e-3), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "index_build_us": build_ms * 1e3, "mask_step_us": mask_ms * 1e3,
+        "walk_kernel_us": walk_ms_mean * 1e3,
+        "config": config_dict(w, world),
+        "roofline": {"bound": "hbm", "kernel": "walk (index build: next-state + bitmask stores)",
+                     "achieved": achieved, "peak": hbm_gbs, "unit": "GB/s",
+                     "frac": achieved / hbm_gbs, "peak_kind": f"of {peak_kind}",
+                     "algorithmic_bytes_per_launch": walk_bytes, "traffic": None},
+        "roofline_mask_step": {"bound": "hbm", "kernel": "mask_step",
+                               "achieved": mask_achieved, "peak": hbm_gbs, "unit": "GB/s",
+                               "frac": mask_achieved / hbm_gbs, "peak_kind": f"of {peak_kind}",
+                               "algorithmic_bytes_per_launch": mask_bytes, "traffic": None},
+        "clocks": clocks,
+        "e2e": {"value": walks * world / e2e_s, "unit": UNIT, "ms_per_step": e2e_s * 1e3,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "note": "host DFA, vocabulary, logits and states copied in, tokens/states/finished "
+                        "copied out, every step; the index stays on the device for its consumer"},
+        "gpu_launches": 5 * args.steps,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(w, starts)
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

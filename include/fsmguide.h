@@ -163,7 +163,22 @@ int guided_mask_step(const void* logits_in, void* logits_out, int32_t logits_dty
 #define FSM_TUNE_MASK_CLUSTER 2     /* CTAs per logits row in guided_mask_step: 1,2,4,8; 0 = auto */
 #define FSM_TUNE_WALK_CTAS 3        /* CTAs of the walk kernel; 0 = one per SM */
 #define FSM_TUNE_SMEM_TABLE_BYTES 4 /* cap on the shared-memory table tile; 0 = device maximum */
+#define FSM_PROFILE_WALK 5          /* non-zero: record a CUDA event pair around the walk
+                                       kernel of every index build (see fsm_profile_read) */
 int fsm_debug_set(int32_t key, int32_t value);
+
+/*
+ * Instrumentation (no counterpart in the paper).  While FSM_PROFILE_WALK is set,
+ * each index build brackets its walk kernel (the launch that produces the
+ * bitmask and the next-state table) with a pair of CUDA events on the build's
+ * stream; nothing is skipped or reordered.  fsm_profile_read synchronises on
+ * the recorded events, writes their elapsed times in milliseconds, oldest
+ * first, to the HOST array ms_out (at most `capacity` values), forgets them and
+ * returns how many it wrote (or FSM_ERR_CUDA).  At most 4096 launches are kept
+ * between reads; later ones are not recorded.  Call it from the thread that
+ * issued the builds, with their device current.
+ */
+int fsm_profile_read(float* ms_out, int32_t capacity);
 
 #ifdef __cplusplus
 }

@@ -15,6 +15,7 @@ import torch
 FSM_STATE_I32, FSM_STATE_U16 = 0, 1
 FSM_LOGITS_F32, FSM_LOGITS_BF16 = 0, 1
 FSM_DEBUG_WEAK_HASH, FSM_TUNE_MASK_CLUSTER, FSM_TUNE_WALK_CTAS, FSM_TUNE_SMEM_TABLE_BYTES = 1, 2, 3, 4
+FSM_PROFILE_WALK = 5
 FSM_FLAG_TRANS_RANGE, FSM_FLAG_OFFSETS, FSM_FLAG_STATE_RANGE = 1, 2, 4
 FSM_FLAG_CLASS_SPLIT, FSM_FLAG_WAIT_TIMEOUT = 8, 16
 
@@ -49,6 +50,8 @@ def lib() -> ctypes.CDLL:
         L.fsm_device_check.restype = ctypes.c_int
         L.fsm_debug_set.argtypes = [i32, i32]
         L.fsm_debug_set.restype = ctypes.c_int
+        L.fsm_profile_read.argtypes = [vp, i32]
+        L.fsm_profile_read.restype = ctypes.c_int
         L.fsm_index_workspace_bytes.argtypes = [i32, i32, i64]
         L.fsm_index_workspace_bytes.restype = sz
         L.fsm_index_build.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, i32, vp, sz, vp, vp]
@@ -87,6 +90,15 @@ def fsm_device_check() -> int:
 
 def fsm_debug_set(key: int, value: int) -> int:
     return lib().fsm_debug_set(key, value)
+
+
+def fsm_profile_read(capacity: int = 4096):
+    """Returns the walk-kernel durations (ms) recorded since the last read."""
+    buf = (ctypes.c_float * capacity)()
+    n = lib().fsm_profile_read(ctypes.cast(buf, ctypes.c_void_p), capacity)
+    if n < 0:
+        raise FsmError(n, "fsm_profile_read")
+    return list(buf[:n])
 
 
 def fsm_index_workspace_bytes(Q: int, N: int, vocab_nbytes: int) -> int:

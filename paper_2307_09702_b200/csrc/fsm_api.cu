@@ -1,4 +1,6 @@
 // Status strings, device query and process-wide knobs of the fsmguide C ABI.
+#include <vector>
+
 #include "fsm_common.cuh"
 
 namespace fsm {
@@ -35,7 +37,58 @@ const DeviceInfo& device_info() {
     return d;
 }
 
+namespace {
+constexpr int kProfileRing = 4096;
+struct EventPair {
+    cudaEvent_t begin, end;
+};
+std::vector<EventPair>& ring() {
+    static std::vector<EventPair> r;
+    return r;
+}
+int g_profile_used = 0;
+}  // namespace
+
+int profile_begin(cudaStream_t stream) {
+    if (!tunables().profile_walk || g_profile_used >= kProfileRing) return -1;
+    std::vector<EventPair>& r = ring();
+    if (g_profile_used >= static_cast<int>(r.size())) {
+        EventPair e;
+        if (cudaEventCreate(&e.begin) != cudaSuccess) return -1;
+        if (cudaEventCreate(&e.end) != cudaSuccess) {
+            cudaEventDestroy(e.begin);
+            return -1;
+        }
+        r.push_back(e);
+    }
+    const int slot = g_profile_used++;
+    cudaEventRecord(r[slot].begin, stream);
+    return slot;
+}
+
+void profile_end(int slot, cudaStream_t stream) {
+    if (slot >= 0) cudaEventRecord(ring()[slot].end, stream);
+}
+
 }  // namespace fsm
+
+extern "C" int fsm_profile_read(float* ms_out, int32_t capacity) {
+    using namespace fsm;
+    int n = 0;
+    int rc = 0;
+    for (int i = 0; i < g_profile_used; ++i) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(ring()[i].end) != cudaSuccess ||
+            cudaEventElapsedTime(&ms, ring()[i].begin, ring()[i].end) != cudaSuccess) {
+            (void)cudaGetLastError();
+            rc = FSM_ERR_CUDA;
+            break;
+        }
+        if (ms_out && n < capacity) ms_out[n++] = ms;
+    }
+    g_profile_used = 0;
+    return rc ? rc : n;
+}
 
 extern "C" const char* fsm_status_string(int status) {
     switch (status) {
@@ -66,6 +119,7 @@ extern "C" int fsm_debug_set(int32_t key, int32_t value) {
         case FSM_TUNE_MASK_CLUSTER: slot = &t.mask_cluster; break;
         case FSM_TUNE_WALK_CTAS: slot = &t.walk_ctas; break;
         case FSM_TUNE_SMEM_TABLE_BYTES: slot = &t.smem_table_cap; break;
+        case FSM_PROFILE_WALK: slot = &t.profile_walk; break;
         default: return FSM_ERR_RANGE;
     }
     int old = *slot;

@@ -20,6 +20,7 @@ struct Tunables {
     int mask_cluster = 0;
     int walk_ctas = 0;
     int smem_table_cap = 0;
+    int profile_walk = 0;
 };
 Tunables& tunables();
 
@@ -31,6 +32,11 @@ struct DeviceInfo {
 };
 // Properties of the current device (queried once per device index, cached).
 const DeviceInfo& device_info();
+
+// Event pairs behind FSM_PROFILE_WALK.  profile_begin returns a slot (or -1 when
+// profiling is off or the ring is full) after recording the first event.
+int profile_begin(cudaStream_t stream);
+void profile_end(int slot, cudaStream_t stream);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

@@ -465,10 +465,12 @@ extern "C" int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* acc
     int64_t grid = (tasks + kWalkWarps - 1) / kWalkWarps;
     if (grid > dev.sm_count) grid = dev.sm_count;
     if (tune.walk_ctas > 0) grid = tune.walk_ctas;
+    const int prof = profile_begin(stream);
     cudaError_t e = wide ? launch_walk_for<int32_t>(p, static_cast<int>(grid), state_dtype,
                                                    next_state != nullptr, stream)
                          : launch_walk_for<uint16_t>(p, static_cast<int>(grid), state_dtype,
                                                     next_state != nullptr, stream);
+    profile_end(prof, stream);
     return e == cudaSuccess ? FSM_OK : FSM_ERR_CUDA;
 }
 
