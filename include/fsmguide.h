@@ -117,6 +117,41 @@ int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* accept,
                          void* cuda_stream);
 
 /*
+ * Index build without caller-provided scratch.  The paper has no counterpart:
+ * this entry point exists for callers that cannot obtain device scratch memory
+ * themselves - a plug-in running inside a host application that has handed the
+ * whole device to its own memory pool, a serving loop in which cudaMalloc (and
+ * the implicit device synchronisation it brings) is forbidden, or a process
+ * that must not grow its footprint after start-up.
+ *
+ * It computes exactly what fsm_index_build computes (same arguments, same
+ * outputs, same status flags), but takes its scratch from a fixed array of
+ * FSM_STATIC_SCRATCH_BYTES that lives inside the library's device image: every
+ * GPU on which the library is loaded holds those bytes until the process
+ * exits.  The call allocates and frees nothing.
+ *
+ *   - Size limit: the build is refused with FSM_ERR_WORKSPACE, before anything is
+ *     enqueued, when fsm_index_workspace_bytes(Q, N, vocab_nbytes) exceeds
+ *     FSM_STATIC_SCRATCH_BYTES (as a guide: about 1,000 states with 60,000
+ *     tokens, or 2,000 states with 30,000 tokens).  Larger problems need
+ *     fsm_index_build and a workspace.
+ *   - First call on each device: the library looks up the device address of its
+ *     scratch array (the device must be current).  Make that first call outside
+ *     any stream capture.
+ *   - The array is shared by every call on that device and still holds the
+ *     previous call's intermediates; the build overwrites every part it reads,
+ *     so nothing has to be cleared in between.  Two calls whose kernels may run
+ *     at the same time on one device (different streams or threads) race on the
+ *     array: serialise them.
+ */
+#define FSM_STATIC_SCRATCH_BYTES (2u << 20)
+int fsm_index_build_static(const int32_t* dfa_trans, const uint8_t* accept,
+                           const uint8_t* vocab_bytes, const int32_t* vocab_offsets,
+                           int64_t vocab_nbytes, int32_t Q, int32_t N, int32_t dead_state,
+                           int32_t eos_id, uint32_t* allowed_mask, void* next_state,
+                           int32_t state_dtype, int32_t* status_word, void* cuda_stream);
+
+/*
  * One step of guided greedy decoding for a batch (paper Algorithm 2, with the
  * greedy selection rule of Section 2.1 in place of the categorical draw).
  *

@@ -16,6 +16,7 @@ FSM_STATE_I32, FSM_STATE_U16 = 0, 1
 FSM_LOGITS_F32, FSM_LOGITS_BF16 = 0, 1
 FSM_DEBUG_WEAK_HASH, FSM_TUNE_MASK_CLUSTER, FSM_TUNE_WALK_CTAS, FSM_TUNE_SMEM_TABLE_BYTES = 1, 2, 3, 4
 FSM_PROFILE_WALK = 5
+FSM_STATIC_SCRATCH_BYTES = 2 << 20
 FSM_FLAG_TRANS_RANGE, FSM_FLAG_OFFSETS, FSM_FLAG_STATE_RANGE = 1, 2, 4
 FSM_FLAG_CLASS_SPLIT, FSM_FLAG_WAIT_TIMEOUT = 8, 16
 
@@ -59,6 +60,8 @@ def lib() -> ctypes.CDLL:
         L.fsm_index_build_rows.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, i32, i32, i32, vp, vp,
                                            i32, vp, sz, vp, vp]
         L.fsm_index_build_rows.restype = ctypes.c_int
+        L.fsm_index_build_static.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, i32, vp, vp]
+        L.fsm_index_build_static.restype = ctypes.c_int
         L.guided_mask_step.argtypes = [vp, vp, i32, i64, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32,
                                        i32, vp, vp]
         L.guided_mask_step.restype = ctypes.c_int
@@ -122,6 +125,18 @@ def fsm_index_build_rows(dfa_trans, accept, vocab_bytes, vocab_offsets, vocab_nb
                                       q_begin, q_end, _ptr(allowed_mask), _ptr(next_state),
                                       state_dtype, _ptr(workspace), workspace_bytes,
                                       _ptr(status_word), _stream(stream))
+
+
+def fsm_index_build_static(dfa_trans, accept, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N,
+                           dead_state, eos_id, allowed_mask, next_state, state_dtype,
+                           status_word=None, stream=None) -> int:
+    """Index build that takes its scratch from the library's built-in device array
+    (``FSM_STATIC_SCRATCH_BYTES``) instead of a caller workspace; for callers that
+    may not allocate device memory.  Same outputs as ``fsm_index_build``."""
+    return lib().fsm_index_build_static(_ptr(dfa_trans), _ptr(accept), _ptr(vocab_bytes),
+                                        _ptr(vocab_offsets), vocab_nbytes, Q, N, dead_state, eos_id,
+                                        _ptr(allowed_mask), _ptr(next_state), state_dtype,
+                                        _ptr(status_word), _stream(stream))
 
 
 def guided_mask_step(logits_in, logits_out, logits_dtype, row_stride, states, finished, tokens_out,

@@ -484,3 +484,53 @@ extern "C" int fsm_index_build(const int32_t* dfa_trans, const uint8_t* accept,
                                 dead_state, eos_id, 0, Q, allowed_mask, next_state, state_dtype,
                                 workspace, workspace_bytes, status_word, cuda_stream);
 }
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free variant: the scratch of the four kernels above lives in this array inside the
+// library's device image instead of in a caller-provided workspace.  In host code the name
+// `g_static_scratch` is only a handle for the runtime, not a device address: the address the
+// kernels need comes from cudaGetSymbolAddress, looked up once per device.
+namespace fsm {
+namespace {
+static __device__ __align__(256) unsigned char g_static_scratch[FSM_STATIC_SCRATCH_BYTES];
+
+// Device address of g_static_scratch on the current device, or nullptr on failure.
+void* static_scratch_address() {
+    constexpr int kMaxDevices = 64;
+    static void* cached[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        return nullptr;
+    }
+    if (cached[dev] == nullptr) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return nullptr;
+        }
+        cached[dev] = ptr;
+    }
+    return cached[dev];
+}
+}  // namespace
+}  // namespace fsm
+
+extern "C" int fsm_index_build_static(const int32_t* dfa_trans, const uint8_t* accept,
+                                      const uint8_t* vocab_bytes, const int32_t* vocab_offsets,
+                                      int64_t vocab_nbytes, int32_t Q, int32_t N,
+                                      int32_t dead_state, int32_t eos_id, uint32_t* allowed_mask,
+                                      void* next_state, int32_t state_dtype, int32_t* status_word,
+                                      void* cuda_stream) {
+    if (Q <= 0 || N <= 0 || vocab_nbytes < 0) return FSM_ERR_SHAPE;
+    const size_t need = fsm_index_workspace_bytes(Q, N, vocab_nbytes);
+    if (need == 0 || need > FSM_STATIC_SCRATCH_BYTES) return FSM_ERR_WORKSPACE;
+    if (!fsm::device_info().ok) return FSM_ERR_CUDA;
+    void* scratch = fsm::static_scratch_address();
+    if (scratch == nullptr) return FSM_ERR_CUDA;
+    // Every part of the scratch that the build reads is written earlier in the same build,
+    // so the previous call's leftovers need no clearing.
+    return fsm_index_build_rows(dfa_trans, accept, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N,
+                                dead_state, eos_id, 0, Q, allowed_mask, next_state, state_dtype,
+                                scratch, FSM_STATIC_SCRATCH_BYTES, status_word, cuda_stream);
+}
