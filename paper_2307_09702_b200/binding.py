@@ -16,6 +16,7 @@ FSM_STATE_I32, FSM_STATE_U16 = 0, 1
 FSM_LOGITS_F32, FSM_LOGITS_BF16 = 0, 1
 FSM_DEBUG_WEAK_HASH, FSM_TUNE_MASK_CLUSTER, FSM_TUNE_WALK_CTAS, FSM_TUNE_SMEM_TABLE_BYTES = 1, 2, 3, 4
 FSM_PROFILE_WALK = 5
+FSM_TUNE_WALK_ALGO = 6
 FSM_STATIC_SCRATCH_BYTES = 2 << 20
 FSM_FLAG_TRANS_RANGE, FSM_FLAG_OFFSETS, FSM_FLAG_STATE_RANGE = 1, 2, 4
 FSM_FLAG_CLASS_SPLIT, FSM_FLAG_WAIT_TIMEOUT = 8, 16

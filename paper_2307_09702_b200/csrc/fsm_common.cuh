@@ -21,6 +21,7 @@ struct Tunables {
     int walk_ctas = 0;
     int smem_table_cap = 0;
     int profile_walk = 0;
+    int walk_algo = 0;
 };
 Tunables& tunables();
 

@@ -25,6 +25,13 @@ constexpr int kWalkWarps = kWalkThreads / 32;
 constexpr int kChunk = 32;             // states per warp task
 constexpr int kInlineBytes = 16;       // token bytes kept in registers
 constexpr uint32_t kBulkChunk = 32768; // bytes per bulk copy instruction
+constexpr int kSeg = 4096;             // tokens per vocabulary segment (bucketed walk)
+constexpr int kSortThreads = 1024;     // threads of the per-segment counting sort
+constexpr int kTeams = 4;              // independent 8-warp teams per CTA (bucketed walk)
+constexpr int kTeamWarps = 8;
+constexpr int kTeamThreads = kTeamWarps * 32;
+constexpr int kBatch = 4;              // 32-token chunks in flight per warp
+constexpr int kBStride = 264;          // bucket-start entries kept per segment (>= 257)
 
 struct IndexMeta {
     int32_t C;        // number of byte classes (the null class has id C)
@@ -41,6 +48,9 @@ struct Workspace {
     void* table;         // [Q][kMaxCs] of TabT (row stride Cs once known)
     uint4* tok_cls;      // [G*32] first 16 class ids of each token
     uint8_t* tok_len;    // [G*32] min(length, 17)
+    uint4* srec;         // [nseg*kSeg] bucket-sorted token records: {min(len,17), class of byte 1..15}
+    uint16_t* slid;      // [nseg*kSeg] token id within its segment, same order as srec
+    uint16_t* bstart;    // [nseg*kBStride] first sorted position of each first-byte class
     size_t bytes;
 };
 
@@ -63,6 +73,10 @@ Workspace carve(void* base, int32_t Q, int32_t N) {
     w.table = take(static_cast<size_t>(Q) * kMaxCs * table_elem_bytes(Q));
     w.tok_cls = reinterpret_cast<uint4*>(take(G * 32 * sizeof(uint4)));
     w.tok_len = take(G * 32);
+    const size_t nseg = (static_cast<size_t>(N) + kSeg - 1) / kSeg;
+    w.srec = reinterpret_cast<uint4*>(take(nseg * kSeg * sizeof(uint4)));
+    w.slid = reinterpret_cast<uint16_t*>(take(nseg * kSeg * sizeof(uint16_t)));
+    w.bstart = reinterpret_cast<uint16_t*>(take(nseg * kBStride * sizeof(uint16_t)));
     w.bytes = off;
     return w;
 }
@@ -99,31 +113,50 @@ __global__ void __launch_bounds__(256) hash_columns(const int32_t* __restrict__ 
 }
 
 // ---------------------------------------------------------------------------- 2
+// One block.  Bytes whose column hashes are equal form a class, represented by the
+// smallest such byte; class ids are the ranks of the representatives.  Equal hashes
+// are found through a small open-addressing table in shared memory.
 __global__ void __launch_bounds__(256) derive_classes(const uint64_t* __restrict__ partial,
                                                      int nblocks, IndexMeta* meta,
                                                      uint8_t* cls, uint8_t* class_rep) {
-    __shared__ uint64_t h[256];
-    __shared__ int rep[256];
+    constexpr int kSlots = 1024;
+    __shared__ unsigned long long keys[kSlots];
+    __shared__ int min_byte[kSlots];
+    __shared__ uint32_t rep_bits[8];
+    constexpr unsigned long long kEmpty = ~0ull;
     const int b = threadIdx.x;
     uint64_t sum = 0;
+#pragma unroll 8
     for (int k = 0; k < nblocks; ++k) sum += partial[k * 256 + b];
-    h[b] = sum;
+    // kEmpty marks a free slot; folding that one value onto its neighbour can only merge
+    // two classes, which the exact verification of the next kernel would catch.
+    const unsigned long long key = (sum == kEmpty) ? sum - 1 : sum;
+    for (int i = b; i < kSlots; i += 256) {
+        keys[i] = kEmpty;
+        min_byte[i] = 256;
+    }
     __syncthreads();
-    int r = b;
-    for (int k = 0; k < b; ++k)
-        if (h[k] == sum) {
-            r = k;
-            break;
-        }
-    rep[b] = r;
+    // at most 256 distinct keys in 1024 slots: linear probing ends within kSlots steps
+    int slot = static_cast<int>((key ^ (key >> 29)) & (kSlots - 1));
+    for (int probe = 0; probe < kSlots; ++probe) {
+        const unsigned long long was = atomicCAS(&keys[slot], kEmpty, key);
+        if (was == kEmpty || was == key) break;
+        slot = (slot + 1) & (kSlots - 1);
+    }
+    atomicMin(&min_byte[slot], b);
     __syncthreads();
-    int id = 0;  // rank of my representative among the representatives
-    for (int k = 0; k < r; ++k) id += (rep[k] == k);
+    const int r = min_byte[slot];
+    const bool is_rep = (r == b);
+    const uint32_t m = __ballot_sync(kFullWarp, is_rep);
+    if ((b & 31) == 0) rep_bits[b >> 5] = m;
+    __syncthreads();
+    int id = __popc(rep_bits[r >> 5] & ((1u << (r & 31)) - 1u));
+    for (int w = 0; w < (r >> 5); ++w) id += __popc(rep_bits[w]);
     cls[b] = static_cast<uint8_t>(id);
-    if (r == b) class_rep[id] = static_cast<uint8_t>(b);
-    int is_rep = (r == b);
-    int C = __syncthreads_count(is_rep);
+    if (is_rep) class_rep[id] = static_cast<uint8_t>(b);
     if (b == 0) {
+        int C = 0;
+        for (int w = 0; w < 8; ++w) C += __popc(rep_bits[w]);
         meta->C = C;
         meta->Cs = (C + 1 + 7) & ~7;
         // 256 distinct columns leave no byte value for the null class: such a table
@@ -202,6 +235,10 @@ struct WalkParams {
     int64_t vocab_nbytes;
     int32_t Q, N, G, dead, eos_id, q_begin, q_end;
     uint32_t smem_cap;  // bytes of dynamic shared memory available for the table tile
+    const uint4* srec;
+    const uint16_t* slid;
+    const uint16_t* bstart;
+    const uint8_t* cls;
     uint32_t* mask;
     void* next;
     int32_t* status;
@@ -213,11 +250,18 @@ __device__ __forceinline__ uint32_t tok_byte(const uint4& t, int i) {
 }
 
 // Walks bytes [from, len) of token v through the uncompressed table.
-__device__ __noinline__ uint32_t raw_walk(const WalkParams& p, uint32_t s, int64_t o0, int64_t o1,
-                                          int from) {
-    for (int64_t i = o0 + from; i < o1 && s != static_cast<uint32_t>(p.dead); ++i)
-        s = clamp_state(p.trans[static_cast<size_t>(s) * 256 + p.vocab_bytes[i]], p.Q, p.dead);
+__device__ __noinline__ uint32_t raw_walk_impl(const int32_t* __restrict__ trans,
+                                               const uint8_t* __restrict__ vocab_bytes, int32_t Q,
+                                               int32_t dead, uint32_t s, int64_t o0, int64_t o1,
+                                               int from) {
+    for (int64_t i = o0 + from; i < o1 && s != static_cast<uint32_t>(dead); ++i)
+        s = clamp_state(trans[static_cast<size_t>(s) * 256 + vocab_bytes[i]], Q, dead);
     return s;
+}
+
+__device__ __forceinline__ uint32_t raw_walk(const WalkParams& p, uint32_t s, int64_t o0,
+                                             int64_t o1, int from) {
+    return raw_walk_impl(p.trans, p.vocab_bytes, p.Q, p.dead, s, o0, o1, from);
 }
 
 template <typename OutT, bool HAS_OUT>
@@ -272,7 +316,7 @@ __device__ __forceinline__ void walk_task(const WalkParams& p, const TabT* __res
 
 // Same task on the uncompressed table (exact fallback after a class split).
 template <typename OutT, bool HAS_OUT>
-__device__ __noinline__ void walk_task_raw(const WalkParams& p, int q0, int nq, int g, int lane) {
+__device__ __forceinline__ void walk_task_raw(const WalkParams& p, int q0, int nq, int g, int lane) {
     const int v = g * 32 + lane;
     int64_t o0 = 0, o1 = 0;
     if (v < p.N && v != p.eos_id) {
@@ -355,6 +399,355 @@ __global__ void __launch_bounds__(kWalkThreads, 1) walk(const WalkParams p) {
     }
 }
 
+
+// ---------------------------------------------------------------------------- 3b
+// Bucketed layout for the work-avoiding walk: the vocabulary is cut into segments of
+// kSeg consecutive token ids; inside a segment the non-empty tokens are grouped by the
+// class of their first byte (counting sort in shared memory).  A record keeps the
+// length and the classes of bytes 1..15; the first byte's class is the bucket.
+__global__ void __launch_bounds__(kSortThreads)
+bucket_tokens(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vocab_offsets,
+              int64_t vocab_nbytes, int32_t N, int32_t eos_id, const IndexMeta* meta,
+              const uint8_t* __restrict__ cls, uint4* __restrict__ srec,
+              uint16_t* __restrict__ slid, uint16_t* __restrict__ bstart, int32_t* status) {
+    constexpr int kPer = kSeg / kSortThreads;
+    __shared__ int hist[257];
+    __shared__ int cursor[257];
+    __shared__ uint8_t s_cls[256];
+    const int seg = blockIdx.x;
+    const int base = seg * kSeg;
+    const int n = min(kSeg, N - base);
+    if (threadIdx.x < 256) s_cls[threadIdx.x] = cls[threadIdx.x];
+    for (int c = threadIdx.x; c < 257; c += kSortThreads) hist[c] = 0;
+    __syncthreads();
+    int64_t start[kPer];
+    int length[kPer];  // 0 = not bucketed (empty, EOS, bad offsets, past the end)
+    int first[kPer];
+    bool bad = false;
+#pragma unroll
+    for (int k = 0; k < kPer; ++k) {
+        const int t = threadIdx.x + k * kSortThreads;
+        const int v = base + t;
+        start[k] = 0;
+        length[k] = 0;
+        first[k] = 0;
+        if (t < n && v != eos_id) {
+            const int64_t o0 = vocab_offsets[v], o1 = vocab_offsets[v + 1];
+            if (o0 < 0 || o1 < o0 || o1 > vocab_nbytes) {
+                bad = true;
+            } else if (o1 > o0) {
+                start[k] = o0;
+                length[k] = static_cast<int>(min(o1 - o0, static_cast<int64_t>(kInlineBytes + 1)));
+                first[k] = s_cls[vocab_bytes[o0]];
+                atomicAdd(&hist[first[k]], 1);
+            }
+        }
+    }
+    if (__syncthreads_or(bad) && threadIdx.x == 0) raise_flag(status, FSM_FLAG_OFFSETS);
+    if (threadIdx.x < 32) {  // exclusive prefix over the 256 counters, 8 per lane
+        int local[8], sum = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            local[i] = sum;
+            sum += hist[threadIdx.x * 8 + i];
+        }
+        int incl = sum;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int o = __shfl_up_sync(kFullWarp, incl, off);
+            if (static_cast<int>(threadIdx.x) >= off) incl += o;
+        }
+        const int excl = incl - sum;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) cursor[threadIdx.x * 8 + i] = excl + local[i];
+        if (threadIdx.x == 31) cursor[256] = incl;
+    }
+    __syncthreads();
+    for (int c = threadIdx.x; c < 257; c += kSortThreads)
+        bstart[seg * kBStride + c] = static_cast<uint16_t>(cursor[c]);
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < kPer; ++k) {
+        if (length[k] == 0) continue;
+        uint32_t w[4] = {static_cast<uint32_t>(length[k]), 0, 0, 0};
+        const int nb = min(length[k], kInlineBytes);
+        for (int i = 1; i < nb; ++i)
+            w[i >> 2] |= static_cast<uint32_t>(s_cls[vocab_bytes[start[k] + i]]) << ((i & 3) * 8);
+        const int pos = atomicAdd(&cursor[first[k]], 1);
+        srec[base + pos] = make_uint4(w[0], w[1], w[2], w[3]);
+        slid[base + pos] = static_cast<uint16_t>(threadIdx.x + k * kSortThreads);
+    }
+}
+
+// ---------------------------------------------------------------------------- 4b
+// Work-avoiding walk.  One persistent CTA per SM; the compressed table is staged in
+// shared memory once (bulk async copy) when it fits.  The CTA's 32 warps form four
+// teams of eight; a team's unit of work is (state q, vocabulary segment).  The team
+// fills the segment's slice of row q with `dead` in shared memory, finds the first-byte
+// classes that q can read (one table lookup per class), walks only the tokens of those
+// buckets (lane = token, several 32-token chunks in flight per warp), scatters the
+// survivors' end states and bitmask bits into the slice, then streams the slice to
+// global memory with coalesced 16-byte stores.  Every (state, token) pair still gets
+// its entry; pairs whose first byte is unreadable are settled by the fill.
+struct LiveBucket {
+    uint32_t s1;      // state after the first byte
+    uint16_t start;   // first sorted position of the bucket
+    uint16_t count;
+};
+
+struct TeamScratch {
+    LiveBucket live[256];
+    uint16_t cpre[260];  // 32-token chunks before each live bucket; [n_live] = total
+    int n_live;
+    int n_chunks;
+};
+
+template <typename OutT, bool HAS_OUT>
+__host__ __device__ constexpr size_t team_bytes() {
+    return (HAS_OUT ? kSeg * sizeof(OutT) : 0) + kSeg / 8 + ((sizeof(TeamScratch) + 15) / 16) * 16;
+}
+
+__device__ __forceinline__ void team_sync(int team) {
+    asm volatile("bar.sync %0, %1;" ::"r"(team + 1), "n"(kTeamThreads) : "memory");
+}
+
+template <typename TabT, typename OutT, bool HAS_OUT, bool FULL>
+__device__ __forceinline__ void bucketed_unit(const WalkParams& p, const TabT* __restrict__ tab,
+                                              int C, int Cs, bool raw, OutT* row, uint32_t* mbits,
+                                              TeamScratch* ts, int team, int r, int seg) {
+    const uint32_t dead = p.dead;
+    const int lane = threadIdx.x & 31;
+    const int tw = (threadIdx.x >> 5) & (kTeamWarps - 1);
+    const int tt = threadIdx.x & (kTeamThreads - 1);
+    const int q = p.q_begin + r;
+    const int base = seg * kSeg;
+    const int n = min(kSeg, p.N - base);
+    constexpr int kVecElems = 16 / sizeof(OutT);
+    auto lookup = [&](uint32_t s, uint32_t c) -> uint32_t {
+        if (FULL) return tab[s * static_cast<uint32_t>(Cs) + c];
+        return __ldg(tab + static_cast<size_t>(s) * Cs + c);
+    };
+
+    // ---- fill
+    if (HAS_OUT) {
+        const uint32_t d = sizeof(OutT) == 2 ? (dead | (dead << 16)) : dead;
+        const uint4 dead16 = make_uint4(d, d, d, d);
+        for (int i = tt; i < kSeg / kVecElems; i += kTeamThreads)
+            reinterpret_cast<uint4*>(row)[i] = dead16;
+    }
+    for (int i = tt; i < kSeg / 32; i += kTeamThreads) mbits[i] = 0;
+    if (tw == 0 && !raw) {
+        int cnt = 0, chunks = 0;
+        const uint16_t* bs = p.bstart + static_cast<size_t>(seg) * kBStride;
+        for (int c0 = 0; c0 < C; c0 += 32) {
+            const int c = c0 + lane;
+            uint32_t s1 = dead;
+            int start = 0, num = 0;
+            if (c < C) {
+                s1 = lookup(q, c);
+                start = bs[c];
+                num = bs[c + 1] - start;
+            }
+            const bool is_live = (s1 != dead) && (num > 0);
+            const uint32_t m = __ballot_sync(kFullWarp, is_live);
+            const int nch = is_live ? (num + 31) >> 5 : 0;
+            int incl = nch;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int o = __shfl_up_sync(kFullWarp, incl, off);
+                if (lane >= off) incl += o;
+            }
+            if (is_live) {
+                const int pos = cnt + __popc(m & ((1u << lane) - 1u));
+                LiveBucket b;
+                b.s1 = s1;
+                b.start = static_cast<uint16_t>(start);
+                b.count = static_cast<uint16_t>(num);
+                ts->live[pos] = b;
+                ts->cpre[pos] = static_cast<uint16_t>(chunks + incl - nch);
+            }
+            cnt += __popc(m);
+            chunks += __shfl_sync(kFullWarp, incl, 31);
+        }
+        if (lane == 0) {
+            ts->n_live = cnt;
+            ts->n_chunks = chunks;
+            ts->cpre[cnt] = static_cast<uint16_t>(chunks);
+        }
+    }
+    team_sync(team);
+
+    // ---- walk the live buckets, kBatch chunks in flight per warp
+    if (!raw) {
+        const int M = ts->n_chunks;
+        int b = 0;
+        for (int g0 = tw; g0 < M; g0 += kTeamWarps * kBatch) {
+            uint4 rec[kBatch];
+            uint32_t lid[kBatch], st[kBatch];
+            bool cont[kBatch], act[kBatch];
+#pragma unroll
+            for (int k = 0; k < kBatch; ++k) {
+                const int g = g0 + k * kTeamWarps;
+                rec[k] = make_uint4(0, 0, 0, 0);
+                lid[k] = 0;
+                st[k] = dead;
+                act[k] = false;
+                if (g < M) {
+                    while (g >= ts->cpre[b + 1]) ++b;
+                    const LiveBucket lb = ts->live[b];
+                    const int i = (g - ts->cpre[b]) * 32 + lane;
+                    st[k] = lb.s1;
+                    if (i < lb.count) {
+                        act[k] = true;
+                        rec[k] = __ldg(p.srec + base + lb.start + i);
+                        lid[k] = p.slid[base + lb.start + i];
+                    }
+                }
+            }
+            bool any_cont = false;
+#pragma unroll
+            for (int k = 0; k < kBatch; ++k) {
+                cont[k] = (rec[k].x & 0xFFu) > 1;
+                any_cont |= cont[k];
+            }
+            if (__any_sync(kFullWarp, any_cont)) {
+#pragma unroll
+                for (int j = 1; j < kInlineBytes; ++j) {
+                    any_cont = false;
+#pragma unroll
+                    for (int k = 0; k < kBatch; ++k) {
+                        if (cont[k]) {
+                            st[k] = lookup(st[k], tok_byte(rec[k], j));
+                            cont[k] = (st[k] != dead) && (j + 1 < static_cast<int>(rec[k].x & 0xFFu));
+                        }
+                        any_cont |= cont[k];
+                    }
+                    if (!__any_sync(kFullWarp, any_cont)) break;
+                }
+#pragma unroll
+                for (int k = 0; k < kBatch; ++k)
+                    if (cont[k]) {  // longer than the inline record: finish on the raw bytes
+                        const int v = base + lid[k];
+                        st[k] = raw_walk(p, st[k], p.vocab_offsets[v], p.vocab_offsets[v + 1],
+                                         kInlineBytes);
+                    }
+            }
+#pragma unroll
+            for (int k = 0; k < kBatch; ++k)
+                if (act[k] && st[k] != dead) {
+                    if (HAS_OUT) row[lid[k]] = static_cast<OutT>(st[k]);
+                    atomicOr(&mbits[lid[k] >> 5], 1u << (lid[k] & 31));
+                }
+        }
+    } else {
+        for (int t = tt; t < n; t += kTeamThreads) {
+            const int v = base + t;
+            if (v == p.eos_id || q == p.dead) continue;
+            const int64_t o0 = p.vocab_offsets[v], o1 = p.vocab_offsets[v + 1];
+            if (o0 < 0 || o1 <= o0 || o1 > p.vocab_nbytes) continue;
+            const uint32_t s = raw_walk(p, q, o0, o1, 0);
+            if (s != dead) {
+                if (HAS_OUT) row[t] = static_cast<OutT>(s);
+                atomicOr(&mbits[t >> 5], 1u << (t & 31));
+            }
+        }
+    }
+    if (tt == 0 && p.eos_id >= base && p.eos_id < base + n && q != p.dead && p.accept[q]) {
+        const int e = p.eos_id - base;
+        if (HAS_OUT) row[e] = static_cast<OutT>(q);
+        atomicOr(&mbits[e >> 5], 1u << (e & 31));
+    }
+    team_sync(team);
+
+    // ---- stream the slice out
+    if (HAS_OUT) {
+        OutT* dst = static_cast<OutT*>(p.next) + static_cast<size_t>(r) * p.N + base;
+        if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+            const int nvec = n / kVecElems;
+            for (int i = tt; i < nvec; i += kTeamThreads)
+                reinterpret_cast<uint4*>(dst)[i] = reinterpret_cast<const uint4*>(row)[i];
+            for (int i = nvec * kVecElems + tt; i < n; i += kTeamThreads) dst[i] = row[i];
+        } else {
+            for (int i = tt; i < n; i += kTeamThreads) dst[i] = row[i];
+        }
+    }
+    uint32_t* mdst = p.mask + static_cast<size_t>(r) * p.G + (base >> 5);
+    for (int i = tt; i < (n + 31) / 32; i += kTeamThreads) mdst[i] = mbits[i];
+    team_sync(team);  // the slice is free for the next unit's fill
+}
+
+template <typename TabT, typename OutT, bool HAS_OUT>
+__global__ void __launch_bounds__(kWalkThreads, 1) walk_bucketed(const WalkParams p) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    __shared__ uint64_t bar;
+    constexpr size_t kTeamBytes = team_bytes<OutT, HAS_OUT>();
+    constexpr size_t kTeamArea = (kTeams * kTeamBytes + 127) / 128 * 128;
+    const int team = threadIdx.x / kTeamThreads;
+    uint8_t* mine = smem_raw + team * kTeamBytes;
+    OutT* row = reinterpret_cast<OutT*>(mine);
+    uint32_t* mbits = reinterpret_cast<uint32_t*>(mine + (HAS_OUT ? kSeg * sizeof(OutT) : 0));
+    TeamScratch* ts = reinterpret_cast<TeamScratch*>(reinterpret_cast<uint8_t*>(mbits) + kSeg / 8);
+    TabT* stab = reinterpret_cast<TabT*>(smem_raw + kTeamArea);
+
+    const TabT* gtab = static_cast<const TabT*>(p.table);
+    const int C = p.meta->C, Cs = p.meta->Cs;
+    const bool raw = p.meta->any_bad != 0;
+    const uint64_t table_bytes = static_cast<uint64_t>(p.Q) * Cs * sizeof(TabT);
+    const bool full = !raw && p.smem_cap > kTeamArea && table_bytes <= p.smem_cap - kTeamArea;
+
+    if (full) {
+        if (threadIdx.x == 0) {
+            mbar_init(&bar, 1);
+            fence_mbar_init();
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const uint32_t bytes = static_cast<uint32_t>(table_bytes);
+            mbar_expect_tx(&bar, bytes);
+            for (uint32_t o = 0; o < bytes; o += kBulkChunk)
+                bulk_copy_g2s(reinterpret_cast<uint8_t*>(stab) + o,
+                              reinterpret_cast<const uint8_t*>(gtab) + o,
+                              min(kBulkChunk, bytes - o), &bar);
+        }
+        bool ok = mbar_wait_bounded(&bar, 0);
+        if (!ok) ok = mbar_wait_bounded(&bar, 0);  // drain before giving up
+        if (!__syncthreads_and(ok)) {
+            if (threadIdx.x == 0) raise_flag(p.status, FSM_FLAG_WAIT_TIMEOUT);
+            return;
+        }
+    }
+
+    const int nseg = (p.N + kSeg - 1) / kSeg;
+    const int64_t units = static_cast<int64_t>(p.q_end - p.q_begin) * nseg;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * kTeams;
+    for (int64_t u = static_cast<int64_t>(blockIdx.x) * kTeams + team; u < units; u += stride) {
+        const int r = static_cast<int>(u / nseg);
+        const int seg = static_cast<int>(u - static_cast<int64_t>(r) * nseg);
+        if (full)
+            bucketed_unit<TabT, OutT, HAS_OUT, true>(p, stab, C, Cs, raw, row, mbits, ts, team, r, seg);
+        else
+            bucketed_unit<TabT, OutT, HAS_OUT, false>(p, gtab, C, Cs, raw, row, mbits, ts, team, r, seg);
+    }
+}
+
+template <typename TabT, typename OutT, bool HAS_OUT>
+cudaError_t launch_bucketed(const WalkParams& p, int grid, cudaStream_t stream) {
+    auto kernel = walk_bucketed<TabT, OutT, HAS_OUT>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(p.smem_cap));
+    if (e != cudaSuccess) return e;
+    kernel<<<grid, kWalkThreads, p.smem_cap, stream>>>(p);
+    return cudaGetLastError();
+}
+
+template <typename TabT>
+cudaError_t launch_bucketed_for(const WalkParams& p, int grid, int32_t state_dtype, bool has_out,
+                                cudaStream_t stream) {
+    if (!has_out) return launch_bucketed<TabT, int32_t, false>(p, grid, stream);
+    if (state_dtype == FSM_STATE_U16) return launch_bucketed<TabT, uint16_t, true>(p, grid, stream);
+    return launch_bucketed<TabT, int32_t, true>(p, grid, stream);
+}
+
 template <typename TabT, typename OutT, bool HAS_OUT>
 cudaError_t launch_walk(const WalkParams& p, int grid, cudaStream_t stream) {
     auto kernel = walk<TabT, OutT, HAS_OUT>;
@@ -422,7 +815,8 @@ extern "C" int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* acc
     derive_classes<<<1, 256, 0, stream>>>(ws.partial, hash_blocks, ws.meta, ws.cls, ws.class_rep);
     const int G = (N + 31) / 32;
     const int row_blocks = Q < 2 * dev.sm_count ? Q : 2 * dev.sm_count;
-    const int tok_blocks = (G * 32 + 255) / 256;
+    const bool bucketed = tune.walk_algo != 1;
+    const int tok_blocks = bucketed ? 0 : (G * 32 + 255) / 256;  // token records of the dense walk
     if (wide)
         prepare_inputs<int32_t><<<row_blocks + tok_blocks, 256, 0, stream>>>(
             dfa_trans, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
@@ -433,6 +827,11 @@ extern "C" int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* acc
             dfa_trans, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
             row_blocks, ws.meta, ws.cls, ws.class_rep, static_cast<uint16_t*>(ws.table),
             ws.tok_cls, ws.tok_len, status_word);
+    const int nseg = (N + kSeg - 1) / kSeg;
+    if (bucketed)
+        bucket_tokens<<<nseg, kSortThreads, 0, stream>>>(vocab_bytes, vocab_offsets, vocab_nbytes,
+                                                          N, eos_id, ws.meta, ws.cls, ws.srec,
+                                                          ws.slid, ws.bstart, status_word);
     if (cudaGetLastError() != cudaSuccess) return FSM_ERR_CUDA;
 
     WalkParams p;
@@ -455,8 +854,28 @@ extern "C" int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* acc
     p.mask = allowed_mask;
     p.next = next_state;
     p.status = status_word;
+    p.srec = ws.srec;
+    p.slid = ws.slid;
+    p.bstart = ws.bstart;
+    p.cls = ws.cls;
     int cap = dev.smem_optin - 1024;  // static shared memory and alignment slack
     if (tune.smem_table_cap > 0 && tune.smem_table_cap < cap) cap = tune.smem_table_cap;
+    if (bucketed) {
+        const int min_cap = static_cast<int>(kTeams * team_bytes<int32_t, true>()) + 256;
+        if (cap < min_cap) cap = min_cap;
+        p.smem_cap = static_cast<uint32_t>(cap) / 128 * 128;
+        const int64_t units = static_cast<int64_t>(q_end - q_begin) * nseg;
+        int64_t grid = dev.sm_count;
+        if (tune.walk_ctas > 0) grid = tune.walk_ctas;
+        if (grid > (units + kTeams - 1) / kTeams) grid = (units + kTeams - 1) / kTeams;
+        const int prof = profile_begin(stream);
+        cudaError_t e = wide ? launch_bucketed_for<int32_t>(p, static_cast<int>(grid), state_dtype,
+                                                           next_state != nullptr, stream)
+                             : launch_bucketed_for<uint16_t>(p, static_cast<int>(grid), state_dtype,
+                                                            next_state != nullptr, stream);
+        profile_end(prof, stream);
+        return e == cudaSuccess ? FSM_OK : FSM_ERR_CUDA;
+    }
     const int min_cap = kChunk * kMaxCs * 4;
     if (cap < min_cap) cap = min_cap;
     p.smem_cap = static_cast<uint32_t>(cap) / 128 * 128;
