@@ -132,8 +132,8 @@ int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* accept,
  *
  *   - Size limit: the build is refused with FSM_ERR_WORKSPACE, before anything is
  *     enqueued, when fsm_index_workspace_bytes(Q, N, vocab_nbytes) exceeds
- *     FSM_STATIC_SCRATCH_BYTES (as a guide: about 1,000 states with 60,000
- *     tokens, or 2,000 states with 30,000 tokens).  Larger problems need
+ *     FSM_STATIC_SCRATCH_BYTES (as a guide: about 1,000 states with 30,000
+ *     tokens, or 2,000 states with 15,000 tokens).  Larger problems need
  *     fsm_index_build and a workspace.
  *   - First call on each device: the library looks up the device address of its
  *     scratch array (the device must be current).  Make that first call outside

@@ -25,13 +25,7 @@ constexpr int kWalkWarps = kWalkThreads / 32;
 constexpr int kChunk = 32;             // states per warp task
 constexpr int kInlineBytes = 16;       // token bytes kept in registers
 constexpr uint32_t kBulkChunk = 32768; // bytes per bulk copy instruction
-constexpr int kSeg = 4096;             // tokens per vocabulary segment (bucketed walk)
-constexpr int kSortThreads = 1024;     // threads of the per-segment counting sort
-constexpr int kTeams = 4;              // independent 8-warp teams per CTA (bucketed walk)
-constexpr int kTeamWarps = 8;
-constexpr int kTeamThreads = kTeamWarps * 32;
-constexpr int kBatch = 4;              // 32-token chunks in flight per warp
-constexpr int kBStride = 264;          // bucket-start entries kept per segment (>= 257)
+constexpr int kBatch = 4;              // 32-token chunks in flight per warp (sparse walk)
 
 struct IndexMeta {
     int32_t C;        // number of byte classes (the null class has id C)
@@ -48,9 +42,11 @@ struct Workspace {
     void* table;         // [Q][kMaxCs] of TabT (row stride Cs once known)
     uint4* tok_cls;      // [G*32] first 16 class ids of each token
     uint8_t* tok_len;    // [G*32] min(length, 17)
-    uint4* srec;         // [nseg*kSeg] bucket-sorted token records: {min(len,17), class of byte 1..15}
-    uint16_t* slid;      // [nseg*kSeg] token id within its segment, same order as srec
-    uint16_t* bstart;    // [nseg*kBStride] first sorted position of each first-byte class
+    uint4* srec;         // [N] tokens sorted by first-byte class: {min(len,17), class of byte 1..15}
+    int32_t* sid;        // [N] token id, same order as srec
+    int32_t* gcount;     // [256] tokens per first-byte class
+    int32_t* gcursor;    // [256] placement cursors of the counting sort
+    int32_t* gstart;     // [257] first sorted position of each class
     size_t bytes;
 };
 
@@ -73,10 +69,11 @@ Workspace carve(void* base, int32_t Q, int32_t N) {
     w.table = take(static_cast<size_t>(Q) * kMaxCs * table_elem_bytes(Q));
     w.tok_cls = reinterpret_cast<uint4*>(take(G * 32 * sizeof(uint4)));
     w.tok_len = take(G * 32);
-    const size_t nseg = (static_cast<size_t>(N) + kSeg - 1) / kSeg;
-    w.srec = reinterpret_cast<uint4*>(take(nseg * kSeg * sizeof(uint4)));
-    w.slid = reinterpret_cast<uint16_t*>(take(nseg * kSeg * sizeof(uint16_t)));
-    w.bstart = reinterpret_cast<uint16_t*>(take(nseg * kBStride * sizeof(uint16_t)));
+    w.srec = reinterpret_cast<uint4*>(take(static_cast<size_t>(N) * sizeof(uint4)));
+    w.sid = reinterpret_cast<int32_t*>(take(static_cast<size_t>(N) * sizeof(int32_t)));
+    w.gcount = reinterpret_cast<int32_t*>(take(256 * sizeof(int32_t)));
+    w.gcursor = reinterpret_cast<int32_t*>(take(256 * sizeof(int32_t)));
+    w.gstart = reinterpret_cast<int32_t*>(take(257 * sizeof(int32_t)));
     w.bytes = off;
     return w;
 }
@@ -118,8 +115,11 @@ __global__ void __launch_bounds__(256) hash_columns(const int32_t* __restrict__ 
 // are found through a small open-addressing table in shared memory.
 __global__ void __launch_bounds__(256) derive_classes(const uint64_t* __restrict__ partial,
                                                      int nblocks, IndexMeta* meta,
-                                                     uint8_t* cls, uint8_t* class_rep) {
+                                                     uint8_t* cls, uint8_t* class_rep,
+                                                     int32_t* gcount, int32_t* gcursor) {
     constexpr int kSlots = 1024;
+    gcount[threadIdx.x] = 0;
+    gcursor[threadIdx.x] = 0;
     __shared__ unsigned long long keys[kSlots];
     __shared__ int min_byte[kSlots];
     __shared__ uint32_t rep_bits[8];
@@ -166,6 +166,31 @@ __global__ void __launch_bounds__(256) derive_classes(const uint64_t* __restrict
     }
 }
 
+// Bounds-checked view of one token for the token-side preparation kernels.
+struct TokenInfo {
+    int64_t start;
+    int len;    // min(length, kInlineBytes + 1); 0 = not bucketed (empty, EOS, bad offsets)
+    int first;  // class of the first byte
+};
+
+__device__ __forceinline__ TokenInfo token_info(const uint8_t* __restrict__ vocab_bytes,
+                                                const int32_t* __restrict__ vocab_offsets,
+                                                int64_t vocab_nbytes, int32_t N, int32_t eos_id,
+                                                const uint8_t* s_cls, int64_t v, bool* bad) {
+    TokenInfo t = {0, 0, 0};
+    if (v < N && v != eos_id) {
+        const int64_t o0 = vocab_offsets[v], o1 = vocab_offsets[v + 1];
+        if (o0 < 0 || o1 < o0 || o1 > vocab_nbytes) {
+            *bad = true;
+        } else if (o1 > o0) {
+            t.start = o0;
+            t.len = static_cast<int>(min(o1 - o0, static_cast<int64_t>(kInlineBytes + 1)));
+            t.first = s_cls[vocab_bytes[o0]];
+        }
+    }
+    return t;
+}
+
 // ---------------------------------------------------------------------------- 3
 // Blocks [0, row_blocks) compress and verify table rows; the remaining blocks
 // translate tokens.  Column C of the compressed table (the null class) and the
@@ -177,7 +202,7 @@ prepare_inputs(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vo
                int32_t N, int32_t dead, int32_t eos_id, int row_blocks, IndexMeta* meta,
                const uint8_t* __restrict__ cls, const uint8_t* __restrict__ class_rep,
                TabT* __restrict__ table, uint4* __restrict__ tok_cls,
-               uint8_t* __restrict__ tok_len, int32_t* status) {
+               uint8_t* __restrict__ tok_len, int32_t* __restrict__ gcount, int32_t* status) {
     const int C = meta->C, Cs = meta->Cs;
     if (static_cast<int>(blockIdx.x) < row_blocks) {
         __shared__ int32_t row[256];
@@ -199,7 +224,21 @@ prepare_inputs(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vo
             atomicExch(&meta->any_bad, 1);
             raise_flag(status, FSM_FLAG_CLASS_SPLIT);
         }
+    } else if (gcount != nullptr) {
+        // sparse walk: count the tokens of each first-byte class (placement: sort_tokens)
+        __shared__ int hist[256];
+        __shared__ uint8_t s_cls[256];
+        hist[threadIdx.x] = 0;
+        s_cls[threadIdx.x] = cls[threadIdx.x];
+        __syncthreads();
+        bool bad = false;
+        const int64_t v = static_cast<int64_t>(blockIdx.x - row_blocks) * 256 + threadIdx.x;
+        const TokenInfo t = token_info(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, s_cls, v, &bad);
+        if (t.len > 0) atomicAdd(&hist[t.first], 1);
+        if (__syncthreads_or(bad) && threadIdx.x == 0) raise_flag(status, FSM_FLAG_OFFSETS);
+        if (hist[threadIdx.x] > 0) atomicAdd(&gcount[threadIdx.x], hist[threadIdx.x]);
     } else {
+        // dense walk: 16-byte class records in token order
         const int64_t slots = (static_cast<int64_t>(N) + 31) / 32 * 32;
         const int64_t v = static_cast<int64_t>(blockIdx.x - row_blocks) * 256 + threadIdx.x;
         if (v >= slots) return;
@@ -236,9 +275,8 @@ struct WalkParams {
     int32_t Q, N, G, dead, eos_id, q_begin, q_end;
     uint32_t smem_cap;  // bytes of dynamic shared memory available for the table tile
     const uint4* srec;
-    const uint16_t* slid;
-    const uint16_t* bstart;
-    const uint8_t* cls;
+    const int32_t* sid;
+    const int32_t* gstart;
     uint32_t* mask;
     void* next;
     int32_t* status;
@@ -401,55 +439,28 @@ __global__ void __launch_bounds__(kWalkThreads, 1) walk(const WalkParams p) {
 
 
 // ---------------------------------------------------------------------------- 3b
-// Bucketed layout for the work-avoiding walk: the vocabulary is cut into segments of
-// kSeg consecutive token ids; inside a segment the non-empty tokens are grouped by the
-// class of their first byte (counting sort in shared memory).  A record keeps the
-// length and the classes of bytes 1..15; the first byte's class is the bucket.
-__global__ void __launch_bounds__(kSortThreads)
-bucket_tokens(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vocab_offsets,
-              int64_t vocab_nbytes, int32_t N, int32_t eos_id, const IndexMeta* meta,
-              const uint8_t* __restrict__ cls, uint4* __restrict__ srec,
-              uint16_t* __restrict__ slid, uint16_t* __restrict__ bstart, int32_t* status) {
-    constexpr int kPer = kSeg / kSortThreads;
-    __shared__ int hist[257];
-    __shared__ int cursor[257];
+// Token order for the work-avoiding walk: all non-empty tokens sorted by the class of
+// their first byte (a counting sort over at most 256 classes).  The per-class counts
+// come from prepare_inputs' token blocks; this kernel places the records.  A record
+// keeps the length and the classes of bytes 1..15 - the first byte's class is the
+// bucket - and `sid` the token id, in the same order.
+__global__ void __launch_bounds__(256)
+sort_tokens(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vocab_offsets,
+            int64_t vocab_nbytes, int32_t N, int32_t eos_id, const uint8_t* __restrict__ cls,
+            const int32_t* __restrict__ gcount, int32_t* __restrict__ gcursor,
+            int32_t* __restrict__ gstart, uint4* __restrict__ srec, int32_t* __restrict__ sid) {
+    __shared__ int lhist[256];
+    __shared__ int lbase[256];
+    __shared__ int gst[257];
     __shared__ uint8_t s_cls[256];
-    const int seg = blockIdx.x;
-    const int base = seg * kSeg;
-    const int n = min(kSeg, N - base);
-    if (threadIdx.x < 256) s_cls[threadIdx.x] = cls[threadIdx.x];
-    for (int c = threadIdx.x; c < 257; c += kSortThreads) hist[c] = 0;
-    __syncthreads();
-    int64_t start[kPer];
-    int length[kPer];  // 0 = not bucketed (empty, EOS, bad offsets, past the end)
-    int first[kPer];
-    bool bad = false;
-#pragma unroll
-    for (int k = 0; k < kPer; ++k) {
-        const int t = threadIdx.x + k * kSortThreads;
-        const int v = base + t;
-        start[k] = 0;
-        length[k] = 0;
-        first[k] = 0;
-        if (t < n && v != eos_id) {
-            const int64_t o0 = vocab_offsets[v], o1 = vocab_offsets[v + 1];
-            if (o0 < 0 || o1 < o0 || o1 > vocab_nbytes) {
-                bad = true;
-            } else if (o1 > o0) {
-                start[k] = o0;
-                length[k] = static_cast<int>(min(o1 - o0, static_cast<int64_t>(kInlineBytes + 1)));
-                first[k] = s_cls[vocab_bytes[o0]];
-                atomicAdd(&hist[first[k]], 1);
-            }
-        }
-    }
-    if (__syncthreads_or(bad) && threadIdx.x == 0) raise_flag(status, FSM_FLAG_OFFSETS);
-    if (threadIdx.x < 32) {  // exclusive prefix over the 256 counters, 8 per lane
+    s_cls[threadIdx.x] = cls[threadIdx.x];
+    lhist[threadIdx.x] = 0;
+    if (threadIdx.x < 32) {  // exclusive prefix over the 256 class counts, 8 per lane
         int local[8], sum = 0;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             local[i] = sum;
-            sum += hist[threadIdx.x * 8 + i];
+            sum += gcount[threadIdx.x * 8 + i];
         }
         int incl = sum;
 #pragma unroll
@@ -457,96 +468,99 @@ bucket_tokens(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict
             const int o = __shfl_up_sync(kFullWarp, incl, off);
             if (static_cast<int>(threadIdx.x) >= off) incl += o;
         }
-        const int excl = incl - sum;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) cursor[threadIdx.x * 8 + i] = excl + local[i];
-        if (threadIdx.x == 31) cursor[256] = incl;
+        for (int i = 0; i < 8; ++i) gst[threadIdx.x * 8 + i] = incl - sum + local[i];
+        if (threadIdx.x == 31) gst[256] = incl;
     }
     __syncthreads();
-    for (int c = threadIdx.x; c < 257; c += kSortThreads)
-        bstart[seg * kBStride + c] = static_cast<uint16_t>(cursor[c]);
+    if (blockIdx.x == 0) {
+        gstart[threadIdx.x] = gst[threadIdx.x];
+        if (threadIdx.x == 0) gstart[256] = gst[256];
+    }
+    bool bad = false;
+    const int64_t v = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
+    const TokenInfo t = token_info(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, s_cls, v, &bad);
+    int rank = 0;
+    if (t.len > 0) rank = atomicAdd(&lhist[t.first], 1);
     __syncthreads();
-#pragma unroll
-    for (int k = 0; k < kPer; ++k) {
-        if (length[k] == 0) continue;
-        uint32_t w[4] = {static_cast<uint32_t>(length[k]), 0, 0, 0};
-        const int nb = min(length[k], kInlineBytes);
+    if (lhist[threadIdx.x] > 0) lbase[threadIdx.x] = atomicAdd(&gcursor[threadIdx.x], lhist[threadIdx.x]);
+    __syncthreads();
+    if (t.len > 0) {
+        uint32_t w[4] = {static_cast<uint32_t>(t.len), 0, 0, 0};
+        const int nb = min(t.len, kInlineBytes);
         for (int i = 1; i < nb; ++i)
-            w[i >> 2] |= static_cast<uint32_t>(s_cls[vocab_bytes[start[k] + i]]) << ((i & 3) * 8);
-        const int pos = atomicAdd(&cursor[first[k]], 1);
-        srec[base + pos] = make_uint4(w[0], w[1], w[2], w[3]);
-        slid[base + pos] = static_cast<uint16_t>(threadIdx.x + k * kSortThreads);
+            w[i >> 2] |= static_cast<uint32_t>(s_cls[vocab_bytes[t.start + i]]) << ((i & 3) * 8);
+        const int pos = gst[t.first] + lbase[t.first] + rank;
+        srec[pos] = make_uint4(w[0], w[1], w[2], w[3]);
+        sid[pos] = static_cast<int32_t>(v);
     }
 }
 
 // ---------------------------------------------------------------------------- 4b
 // Work-avoiding walk.  One persistent CTA per SM; the compressed table is staged in
-// shared memory once (bulk async copy) when it fits.  The CTA's 32 warps form four
-// teams of eight; a team's unit of work is (state q, vocabulary segment).  The team
-// fills the segment's slice of row q with `dead` in shared memory, finds the first-byte
-// classes that q can read (one table lookup per class), walks only the tokens of those
-// buckets (lane = token, several 32-token chunks in flight per warp), scatters the
-// survivors' end states and bitmask bits into the slice, then streams the slice to
-// global memory with coalesced 16-byte stores.  Every (state, token) pair still gets
-// its entry; pairs whose first byte is unreadable are settled by the fill.
+// shared memory once (bulk async copy) when it fits.  A CTA's unit of work is one index
+// row (one state q):
+//   fill     the row of the next-state table is set to `dead` and the bitmask row to 0
+//            with streaming 16-byte stores - this settles every token whose first byte
+//            q cannot read, with no table lookup at all;
+//   buckets  one lookup per byte class tells which first-byte buckets are readable;
+//   walk     only the tokens of those buckets are walked (lane = token, 32-token chunks,
+//            several chunks in flight per warp); survivors store their end state into
+//            the row and OR their bit into the bitmask row.  The row was written
+//            microseconds earlier by the same CTA, so these stores merge in L2 and each
+//            line still reaches HBM once.
+// Every (state, token) pair gets its entry; results are identical to the dense walk.
 struct LiveBucket {
-    uint32_t s1;      // state after the first byte
-    uint16_t start;   // first sorted position of the bucket
-    uint16_t count;
+    uint32_t s1;  // state after the first byte
+    int32_t start;
+    int32_t count;
 };
 
-struct TeamScratch {
-    LiveBucket live[256];
-    uint16_t cpre[260];  // 32-token chunks before each live bucket; [n_live] = total
-    int n_live;
-    int n_chunks;
-};
-
-template <typename OutT, bool HAS_OUT>
-__host__ __device__ constexpr size_t team_bytes() {
-    return (HAS_OUT ? kSeg * sizeof(OutT) : 0) + kSeg / 8 + ((sizeof(TeamScratch) + 15) / 16) * 16;
-}
-
-__device__ __forceinline__ void team_sync(int team) {
-    asm volatile("bar.sync %0, %1;" ::"r"(team + 1), "n"(kTeamThreads) : "memory");
-}
+constexpr int kMaxLive = 256;
 
 template <typename TabT, typename OutT, bool HAS_OUT, bool FULL>
-__device__ __forceinline__ void bucketed_unit(const WalkParams& p, const TabT* __restrict__ tab,
-                                              int C, int Cs, bool raw, OutT* row, uint32_t* mbits,
-                                              TeamScratch* ts, int team, int r, int seg) {
+__device__ __forceinline__ void sparse_row(const WalkParams& p, const TabT* __restrict__ tab,
+                                           int C, int Cs, bool raw, LiveBucket* live,
+                                           int32_t* cpre, int* counts, const int32_t* s_gstart,
+                                           int r) {
     const uint32_t dead = p.dead;
-    const int lane = threadIdx.x & 31;
-    const int tw = (threadIdx.x >> 5) & (kTeamWarps - 1);
-    const int tt = threadIdx.x & (kTeamThreads - 1);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int q = p.q_begin + r;
-    const int base = seg * kSeg;
-    const int n = min(kSeg, p.N - base);
-    constexpr int kVecElems = 16 / sizeof(OutT);
+    OutT* nrow = HAS_OUT ? static_cast<OutT*>(p.next) + static_cast<size_t>(r) * p.N : nullptr;
+    uint32_t* mrow = p.mask + static_cast<size_t>(r) * p.G;
     auto lookup = [&](uint32_t s, uint32_t c) -> uint32_t {
         if (FULL) return tab[s * static_cast<uint32_t>(Cs) + c];
         return __ldg(tab + static_cast<size_t>(s) * Cs + c);
     };
 
-    // ---- fill
+    // ---- fill (head and tail element-wise, the aligned middle as 16-byte vectors)
     if (HAS_OUT) {
+        constexpr int kVecElems = 16 / sizeof(OutT);
+        const uintptr_t addr = reinterpret_cast<uintptr_t>(nrow);
+        int head = static_cast<int>(((16 - (addr & 15)) & 15) / sizeof(OutT));
+        if (head > p.N) head = p.N;
+        const int nvec = (p.N - head) / kVecElems;
         const uint32_t d = sizeof(OutT) == 2 ? (dead | (dead << 16)) : dead;
         const uint4 dead16 = make_uint4(d, d, d, d);
-        for (int i = tt; i < kSeg / kVecElems; i += kTeamThreads)
-            reinterpret_cast<uint4*>(row)[i] = dead16;
+        uint4* mid = reinterpret_cast<uint4*>(nrow + head);
+        for (int i = threadIdx.x; i < nvec; i += kWalkThreads) mid[i] = dead16;
+        for (int i = threadIdx.x; i < head; i += kWalkThreads) nrow[i] = static_cast<OutT>(dead);
+        for (int i = head + nvec * kVecElems + threadIdx.x; i < p.N; i += kWalkThreads)
+            nrow[i] = static_cast<OutT>(dead);
     }
-    for (int i = tt; i < kSeg / 32; i += kTeamThreads) mbits[i] = 0;
-    if (tw == 0 && !raw) {
+    for (int i = threadIdx.x; i < p.G; i += kWalkThreads) mrow[i] = 0;
+
+    // ---- readable buckets of this state
+    if (warp == 0 && !raw) {
         int cnt = 0, chunks = 0;
-        const uint16_t* bs = p.bstart + static_cast<size_t>(seg) * kBStride;
         for (int c0 = 0; c0 < C; c0 += 32) {
             const int c = c0 + lane;
             uint32_t s1 = dead;
             int start = 0, num = 0;
             if (c < C) {
                 s1 = lookup(q, c);
-                start = bs[c];
-                num = bs[c + 1] - start;
+                start = s_gstart[c];
+                num = s_gstart[c + 1] - start;
             }
             const bool is_live = (s1 != dead) && (num > 0);
             const uint32_t m = __ballot_sync(kFullWarp, is_live);
@@ -561,46 +575,46 @@ __device__ __forceinline__ void bucketed_unit(const WalkParams& p, const TabT* _
                 const int pos = cnt + __popc(m & ((1u << lane) - 1u));
                 LiveBucket b;
                 b.s1 = s1;
-                b.start = static_cast<uint16_t>(start);
-                b.count = static_cast<uint16_t>(num);
-                ts->live[pos] = b;
-                ts->cpre[pos] = static_cast<uint16_t>(chunks + incl - nch);
+                b.start = start;
+                b.count = num;
+                live[pos] = b;
+                cpre[pos] = chunks + incl - nch;
             }
             cnt += __popc(m);
             chunks += __shfl_sync(kFullWarp, incl, 31);
         }
         if (lane == 0) {
-            ts->n_live = cnt;
-            ts->n_chunks = chunks;
-            ts->cpre[cnt] = static_cast<uint16_t>(chunks);
+            counts[0] = cnt;
+            counts[1] = chunks;
+            cpre[cnt] = chunks;
         }
     }
-    team_sync(team);
+    __syncthreads();  // also orders the fill before the scattered stores below
 
-    // ---- walk the live buckets, kBatch chunks in flight per warp
     if (!raw) {
-        const int M = ts->n_chunks;
+        const int M = counts[1];
         int b = 0;
-        for (int g0 = tw; g0 < M; g0 += kTeamWarps * kBatch) {
+        for (int g0 = warp; g0 < M; g0 += kWalkWarps * kBatch) {
             uint4 rec[kBatch];
-            uint32_t lid[kBatch], st[kBatch];
+            int32_t id[kBatch];
+            uint32_t st[kBatch];
             bool cont[kBatch], act[kBatch];
 #pragma unroll
             for (int k = 0; k < kBatch; ++k) {
-                const int g = g0 + k * kTeamWarps;
+                const int g = g0 + k * kWalkWarps;
                 rec[k] = make_uint4(0, 0, 0, 0);
-                lid[k] = 0;
+                id[k] = 0;
                 st[k] = dead;
                 act[k] = false;
                 if (g < M) {
-                    while (g >= ts->cpre[b + 1]) ++b;
-                    const LiveBucket lb = ts->live[b];
-                    const int i = (g - ts->cpre[b]) * 32 + lane;
+                    while (g >= cpre[b + 1]) ++b;
+                    const LiveBucket lb = live[b];
+                    const int i = (g - cpre[b]) * 32 + lane;
                     st[k] = lb.s1;
                     if (i < lb.count) {
                         act[k] = true;
-                        rec[k] = __ldg(p.srec + base + lb.start + i);
-                        lid[k] = p.slid[base + lb.start + i];
+                        rec[k] = __ldg(p.srec + lb.start + i);
+                        id[k] = __ldg(p.sid + lb.start + i);
                     }
                 }
             }
@@ -626,75 +640,53 @@ __device__ __forceinline__ void bucketed_unit(const WalkParams& p, const TabT* _
                 }
 #pragma unroll
                 for (int k = 0; k < kBatch; ++k)
-                    if (cont[k]) {  // longer than the inline record: finish on the raw bytes
-                        const int v = base + lid[k];
-                        st[k] = raw_walk(p, st[k], p.vocab_offsets[v], p.vocab_offsets[v + 1],
+                    if (cont[k])  // longer than the inline record: finish on the raw bytes
+                        st[k] = raw_walk(p, st[k], p.vocab_offsets[id[k]], p.vocab_offsets[id[k] + 1],
                                          kInlineBytes);
-                    }
             }
 #pragma unroll
             for (int k = 0; k < kBatch; ++k)
                 if (act[k] && st[k] != dead) {
-                    if (HAS_OUT) row[lid[k]] = static_cast<OutT>(st[k]);
-                    atomicOr(&mbits[lid[k] >> 5], 1u << (lid[k] & 31));
+                    if (HAS_OUT) nrow[id[k]] = static_cast<OutT>(st[k]);
+                    atomicOr(&mrow[id[k] >> 5], 1u << (id[k] & 31));
                 }
         }
-    } else {
-        for (int t = tt; t < n; t += kTeamThreads) {
-            const int v = base + t;
-            if (v == p.eos_id || q == p.dead) continue;
+    } else if (q != p.dead) {
+        for (int v = threadIdx.x; v < p.N; v += kWalkThreads) {
+            if (v == p.eos_id) continue;
             const int64_t o0 = p.vocab_offsets[v], o1 = p.vocab_offsets[v + 1];
             if (o0 < 0 || o1 <= o0 || o1 > p.vocab_nbytes) continue;
             const uint32_t s = raw_walk(p, q, o0, o1, 0);
             if (s != dead) {
-                if (HAS_OUT) row[t] = static_cast<OutT>(s);
-                atomicOr(&mbits[t >> 5], 1u << (t & 31));
+                if (HAS_OUT) nrow[v] = static_cast<OutT>(s);
+                atomicOr(&mrow[v >> 5], 1u << (v & 31));
             }
         }
     }
-    if (tt == 0 && p.eos_id >= base && p.eos_id < base + n && q != p.dead && p.accept[q]) {
-        const int e = p.eos_id - base;
-        if (HAS_OUT) row[e] = static_cast<OutT>(q);
-        atomicOr(&mbits[e >> 5], 1u << (e & 31));
+    if (threadIdx.x == 0 && p.eos_id >= 0 && q != p.dead && p.accept[q]) {
+        if (HAS_OUT) nrow[p.eos_id] = static_cast<OutT>(q);
+        atomicOr(&mrow[p.eos_id >> 5], 1u << (p.eos_id & 31));
     }
-    team_sync(team);
-
-    // ---- stream the slice out
-    if (HAS_OUT) {
-        OutT* dst = static_cast<OutT*>(p.next) + static_cast<size_t>(r) * p.N + base;
-        if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
-            const int nvec = n / kVecElems;
-            for (int i = tt; i < nvec; i += kTeamThreads)
-                reinterpret_cast<uint4*>(dst)[i] = reinterpret_cast<const uint4*>(row)[i];
-            for (int i = nvec * kVecElems + tt; i < n; i += kTeamThreads) dst[i] = row[i];
-        } else {
-            for (int i = tt; i < n; i += kTeamThreads) dst[i] = row[i];
-        }
-    }
-    uint32_t* mdst = p.mask + static_cast<size_t>(r) * p.G + (base >> 5);
-    for (int i = tt; i < (n + 31) / 32; i += kTeamThreads) mdst[i] = mbits[i];
-    team_sync(team);  // the slice is free for the next unit's fill
+    __syncthreads();  // the bucket list is rebuilt by the next row
 }
 
 template <typename TabT, typename OutT, bool HAS_OUT>
-__global__ void __launch_bounds__(kWalkThreads, 1) walk_bucketed(const WalkParams p) {
+__global__ void __launch_bounds__(kWalkThreads, 1) walk_sparse(const WalkParams p) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     __shared__ uint64_t bar;
-    constexpr size_t kTeamBytes = team_bytes<OutT, HAS_OUT>();
-    constexpr size_t kTeamArea = (kTeams * kTeamBytes + 127) / 128 * 128;
-    const int team = threadIdx.x / kTeamThreads;
-    uint8_t* mine = smem_raw + team * kTeamBytes;
-    OutT* row = reinterpret_cast<OutT*>(mine);
-    uint32_t* mbits = reinterpret_cast<uint32_t*>(mine + (HAS_OUT ? kSeg * sizeof(OutT) : 0));
-    TeamScratch* ts = reinterpret_cast<TeamScratch*>(reinterpret_cast<uint8_t*>(mbits) + kSeg / 8);
-    TabT* stab = reinterpret_cast<TabT*>(smem_raw + kTeamArea);
+    __shared__ LiveBucket live[kMaxLive];
+    __shared__ int32_t cpre[kMaxLive + 4];
+    __shared__ int32_t s_gstart[260];
+    __shared__ int counts[2];
+    TabT* stab = reinterpret_cast<TabT*>(smem_raw);
 
     const TabT* gtab = static_cast<const TabT*>(p.table);
     const int C = p.meta->C, Cs = p.meta->Cs;
     const bool raw = p.meta->any_bad != 0;
     const uint64_t table_bytes = static_cast<uint64_t>(p.Q) * Cs * sizeof(TabT);
-    const bool full = !raw && p.smem_cap > kTeamArea && table_bytes <= p.smem_cap - kTeamArea;
+    const bool full = !raw && table_bytes <= p.smem_cap;
 
+    for (int i = threadIdx.x; i < 257; i += kWalkThreads) s_gstart[i] = p.gstart[i];
     if (full) {
         if (threadIdx.x == 0) {
             mbar_init(&bar, 1);
@@ -705,8 +697,7 @@ __global__ void __launch_bounds__(kWalkThreads, 1) walk_bucketed(const WalkParam
             const uint32_t bytes = static_cast<uint32_t>(table_bytes);
             mbar_expect_tx(&bar, bytes);
             for (uint32_t o = 0; o < bytes; o += kBulkChunk)
-                bulk_copy_g2s(reinterpret_cast<uint8_t*>(stab) + o,
-                              reinterpret_cast<const uint8_t*>(gtab) + o,
+                bulk_copy_g2s(smem_raw + o, reinterpret_cast<const uint8_t*>(gtab) + o,
                               min(kBulkChunk, bytes - o), &bar);
         }
         bool ok = mbar_wait_bounded(&bar, 0);
@@ -715,24 +706,22 @@ __global__ void __launch_bounds__(kWalkThreads, 1) walk_bucketed(const WalkParam
             if (threadIdx.x == 0) raise_flag(p.status, FSM_FLAG_WAIT_TIMEOUT);
             return;
         }
+    } else {
+        __syncthreads();
     }
 
-    const int nseg = (p.N + kSeg - 1) / kSeg;
-    const int64_t units = static_cast<int64_t>(p.q_end - p.q_begin) * nseg;
-    const int64_t stride = static_cast<int64_t>(gridDim.x) * kTeams;
-    for (int64_t u = static_cast<int64_t>(blockIdx.x) * kTeams + team; u < units; u += stride) {
-        const int r = static_cast<int>(u / nseg);
-        const int seg = static_cast<int>(u - static_cast<int64_t>(r) * nseg);
+    const int nrows = p.q_end - p.q_begin;
+    for (int r = blockIdx.x; r < nrows; r += gridDim.x) {
         if (full)
-            bucketed_unit<TabT, OutT, HAS_OUT, true>(p, stab, C, Cs, raw, row, mbits, ts, team, r, seg);
+            sparse_row<TabT, OutT, HAS_OUT, true>(p, stab, C, Cs, raw, live, cpre, counts, s_gstart, r);
         else
-            bucketed_unit<TabT, OutT, HAS_OUT, false>(p, gtab, C, Cs, raw, row, mbits, ts, team, r, seg);
+            sparse_row<TabT, OutT, HAS_OUT, false>(p, gtab, C, Cs, raw, live, cpre, counts, s_gstart, r);
     }
 }
 
 template <typename TabT, typename OutT, bool HAS_OUT>
-cudaError_t launch_bucketed(const WalkParams& p, int grid, cudaStream_t stream) {
-    auto kernel = walk_bucketed<TabT, OutT, HAS_OUT>;
+cudaError_t launch_sparse(const WalkParams& p, int grid, cudaStream_t stream) {
+    auto kernel = walk_sparse<TabT, OutT, HAS_OUT>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(p.smem_cap));
     if (e != cudaSuccess) return e;
@@ -741,11 +730,11 @@ cudaError_t launch_bucketed(const WalkParams& p, int grid, cudaStream_t stream) 
 }
 
 template <typename TabT>
-cudaError_t launch_bucketed_for(const WalkParams& p, int grid, int32_t state_dtype, bool has_out,
-                                cudaStream_t stream) {
-    if (!has_out) return launch_bucketed<TabT, int32_t, false>(p, grid, stream);
-    if (state_dtype == FSM_STATE_U16) return launch_bucketed<TabT, uint16_t, true>(p, grid, stream);
-    return launch_bucketed<TabT, int32_t, true>(p, grid, stream);
+cudaError_t launch_sparse_for(const WalkParams& p, int grid, int32_t state_dtype, bool has_out,
+                              cudaStream_t stream) {
+    if (!has_out) return launch_sparse<TabT, int32_t, false>(p, grid, stream);
+    if (state_dtype == FSM_STATE_U16) return launch_sparse<TabT, uint16_t, true>(p, grid, stream);
+    return launch_sparse<TabT, int32_t, true>(p, grid, stream);
 }
 
 template <typename TabT, typename OutT, bool HAS_OUT>
@@ -812,26 +801,27 @@ extern "C" int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* acc
     const int hash_blocks = Q < kHashBlocks ? Q : kHashBlocks;
     hash_columns<<<hash_blocks, 256, 0, stream>>>(dfa_trans, Q, dead_state, ws.partial,
                                                   tune.weak_hash, status_word);
-    derive_classes<<<1, 256, 0, stream>>>(ws.partial, hash_blocks, ws.meta, ws.cls, ws.class_rep);
+    derive_classes<<<1, 256, 0, stream>>>(ws.partial, hash_blocks, ws.meta, ws.cls, ws.class_rep,
+                                          ws.gcount, ws.gcursor);
     const int G = (N + 31) / 32;
     const int row_blocks = Q < 2 * dev.sm_count ? Q : 2 * dev.sm_count;
     const bool bucketed = tune.walk_algo != 1;
-    const int tok_blocks = bucketed ? 0 : (G * 32 + 255) / 256;  // token records of the dense walk
+    const int tok_blocks = (G * 32 + 255) / 256;  // dense: token records; sparse: class counts
+    int32_t* count_into = bucketed ? ws.gcount : nullptr;
     if (wide)
         prepare_inputs<int32_t><<<row_blocks + tok_blocks, 256, 0, stream>>>(
             dfa_trans, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
             row_blocks, ws.meta, ws.cls, ws.class_rep, static_cast<int32_t*>(ws.table),
-            ws.tok_cls, ws.tok_len, status_word);
+            ws.tok_cls, ws.tok_len, count_into, status_word);
     else
         prepare_inputs<uint16_t><<<row_blocks + tok_blocks, 256, 0, stream>>>(
             dfa_trans, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
             row_blocks, ws.meta, ws.cls, ws.class_rep, static_cast<uint16_t*>(ws.table),
-            ws.tok_cls, ws.tok_len, status_word);
-    const int nseg = (N + kSeg - 1) / kSeg;
+            ws.tok_cls, ws.tok_len, count_into, status_word);
     if (bucketed)
-        bucket_tokens<<<nseg, kSortThreads, 0, stream>>>(vocab_bytes, vocab_offsets, vocab_nbytes,
-                                                          N, eos_id, ws.meta, ws.cls, ws.srec,
-                                                          ws.slid, ws.bstart, status_word);
+        sort_tokens<<<(N + 255) / 256, 256, 0, stream>>>(vocab_bytes, vocab_offsets, vocab_nbytes, N,
+                                                         eos_id, ws.cls, ws.gcount, ws.gcursor,
+                                                         ws.gstart, ws.srec, ws.sid);
     if (cudaGetLastError() != cudaSuccess) return FSM_ERR_CUDA;
 
     WalkParams p;
@@ -855,23 +845,21 @@ extern "C" int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* acc
     p.next = next_state;
     p.status = status_word;
     p.srec = ws.srec;
-    p.slid = ws.slid;
-    p.bstart = ws.bstart;
-    p.cls = ws.cls;
+    p.sid = ws.sid;
+    p.gstart = ws.gstart;
     int cap = dev.smem_optin - 1024;  // static shared memory and alignment slack
     if (tune.smem_table_cap > 0 && tune.smem_table_cap < cap) cap = tune.smem_table_cap;
     if (bucketed) {
-        const int min_cap = static_cast<int>(kTeams * team_bytes<int32_t, true>()) + 256;
-        if (cap < min_cap) cap = min_cap;
+        cap -= 8 * 1024;  // static shared memory of walk_sparse (bucket list)
+        if (cap < 1024) cap = 1024;
         p.smem_cap = static_cast<uint32_t>(cap) / 128 * 128;
-        const int64_t units = static_cast<int64_t>(q_end - q_begin) * nseg;
         int64_t grid = dev.sm_count;
         if (tune.walk_ctas > 0) grid = tune.walk_ctas;
-        if (grid > (units + kTeams - 1) / kTeams) grid = (units + kTeams - 1) / kTeams;
+        if (grid > q_end - q_begin) grid = q_end - q_begin;
         const int prof = profile_begin(stream);
-        cudaError_t e = wide ? launch_bucketed_for<int32_t>(p, static_cast<int>(grid), state_dtype,
+        cudaError_t e = wide ? launch_sparse_for<int32_t>(p, static_cast<int>(grid), state_dtype,
                                                            next_state != nullptr, stream)
-                             : launch_bucketed_for<uint16_t>(p, static_cast<int>(grid), state_dtype,
+                             : launch_sparse_for<uint16_t>(p, static_cast<int>(grid), state_dtype,
                                                             next_state != nullptr, stream);
         profile_end(prof, stream);
         return e == cudaSuccess ? FSM_OK : FSM_ERR_CUDA;
