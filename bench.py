@@ -223,6 +223,7 @@ def run_ours(args):
     if fg.fsm_device_check() != 0:
         raise SystemExit("bench.py needs a compute-capability 10.x device")
     dev = torch.device("cuda", local)
+    fg.fsm_debug_set(binding.FSM_TUNE_WALK_ALGO, args.walk_algo)
     w, starts = workload(rank)
     d = w.dfa
     idx = fg.GuidedIndex(d.trans, d.accept, w.vocab_bytes, w.vocab_offsets, d.dead, w.eos_id,
@@ -374,6 +375,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--walk-algo", type=int, default=0, choices=[0, 1, 2],
+                    help="index walk kernel: 0 automatic, 1 dense warp-tile, 2 work-avoiding")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

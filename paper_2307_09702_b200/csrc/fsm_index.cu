@@ -310,10 +310,37 @@ __device__ __forceinline__ void emit(const WalkParams& p, int q, int g, int v, i
     if (lane == 0) p.mask[r * p.G + g] = word;
 }
 
+// Bytes 1.. of one token walked from state s, all 32 lanes in lock step.  `go` says
+// whether this lane still has a live walk with bytes left.  The loop is warp-uniform
+// (one vote per byte) and its body has no branches: lanes that are done keep their
+// state through a select.  Every state value is a valid table row (out-of-range
+// entries were replaced by `dead` when the table was compressed), so the shared-memory
+// lookup needs no guard; the global-memory lookup is predicated to save traffic.
+template <typename TabT, bool FULL>
+__device__ __forceinline__ uint32_t walk_rest(const TabT* __restrict__ tab, uint32_t Cs,
+                                              uint32_t dead, const uint4& tk, int len, uint32_t s,
+                                              bool& go) {
+#pragma unroll
+    for (int i = 1; i < kInlineBytes; ++i) {
+        if (!__any_sync(kFullWarp, go)) break;
+        const uint32_t c = tok_byte(tk, i);
+        uint32_t ns;
+        if (FULL) {
+            ns = tab[s * Cs + c];
+        } else {
+            ns = s;
+            if (go) ns = __ldg(tab + static_cast<size_t>(s) * Cs + c);
+        }
+        s = go ? ns : s;
+        go = go && (ns != dead) && (i + 1 < len);
+    }
+    return s;
+}
+
 // One warp task: tokens 32g .. 32g+31 (lane = token) from states q0 .. q0+nq-1.
 // `first` points at row q0 of the shared-memory tile; `tab` is the table used for
 // the second and later bytes (the same tile when FULL, else global memory).
-template <typename TabT, typename OutT, bool HAS_OUT, bool FULL>
+template <typename TabT, typename OutT, bool HAS_OUT, bool FULL, bool HAS_EOS>
 __device__ __forceinline__ void walk_task(const WalkParams& p, const TabT* __restrict__ first,
                                           const TabT* __restrict__ tab, int Cs, int q0, int nq,
                                           int g, int lane) {
@@ -322,33 +349,28 @@ __device__ __forceinline__ void walk_task(const WalkParams& p, const TabT* __res
     const int len = p.tok_len[v];
     const uint32_t dead = p.dead;
     const bool multi = len > 1;
-    const bool has_eos = (p.eos_id >= 0) && ((p.eos_id >> 5) == g);
-    const bool eos_lane = (v == p.eos_id);
+    const bool eos_lane = HAS_EOS && (v == p.eos_id);
+    const bool store_ok = HAS_OUT && (v < p.N);
     const TabT* f = first + (tk.x & 0xFFu);
+    const size_t r0 = static_cast<size_t>(q0 - p.q_begin);
+    OutT* outp = HAS_OUT ? static_cast<OutT*>(p.next) + r0 * p.N + v : nullptr;
+    uint32_t* mp = p.mask + r0 * p.G + g;
     for (int j = 0; j < nq; ++j) {
-        const int q = q0 + j;
-        uint32_t s = f[static_cast<size_t>(j) * Cs];
-        bool cont = multi && (s != dead);
-        if (__any_sync(kFullWarp, cont)) {
-#pragma unroll
-            for (int i = 1; i < kInlineBytes; ++i) {
-                if (cont) {
-                    const uint32_t c = tok_byte(tk, i);
-                    if (FULL)
-                        s = tab[s * static_cast<uint32_t>(Cs) + c];
-                    else
-                        s = __ldg(tab + static_cast<size_t>(s) * Cs + c);
-                    cont = (s != dead) && (i + 1 < len);
-                }
-                if (!__any_sync(kFullWarp, cont)) break;
-            }
-            if (cont) {  // longer than the inline record: finish on the raw bytes
-                const int64_t o0 = p.vocab_offsets[v], o1 = p.vocab_offsets[v + 1];
-                s = raw_walk(p, s, o0, o1, kInlineBytes);
-            }
+        uint32_t s = *f;
+        bool go = multi && (s != dead);
+        s = walk_rest<TabT, FULL>(tab, Cs, dead, tk, len, s, go);
+        if (go)  // longer than the inline record and still alive: finish on the raw bytes
+            s = raw_walk(p, s, p.vocab_offsets[v], p.vocab_offsets[v + 1], kInlineBytes);
+        if (HAS_EOS) {
+            const int q = q0 + j;
+            if (eos_lane) s = (q != p.dead && p.accept[q]) ? q : dead;
         }
-        if (has_eos && eos_lane) s = (q != p.dead && p.accept[q]) ? q : dead;
-        emit<OutT, HAS_OUT>(p, q, g, v, lane, s);
+        if (store_ok) *outp = static_cast<OutT>(s);
+        const uint32_t word = __ballot_sync(kFullWarp, s != dead);
+        if (lane == 0) *mp = word;
+        f += Cs;
+        if (HAS_OUT) outp += p.N;
+        mp += p.G;
     }
 }
 
@@ -428,10 +450,17 @@ __global__ void __launch_bounds__(kWalkThreads, 1) walk(const WalkParams p) {
                 walk_task_raw<OutT, HAS_OUT>(p, q0, nq, g, lane);
             } else {
                 const TabT* first = tile + static_cast<size_t>(q0 - t_q0) * Cs;
-                if (full)
-                    walk_task<TabT, OutT, HAS_OUT, true>(p, first, tile, Cs, q0, nq, g, lane);
-                else
-                    walk_task<TabT, OutT, HAS_OUT, false>(p, first, gtab, Cs, q0, nq, g, lane);
+                const bool has_eos = (p.eos_id >= 0) && ((p.eos_id >> 5) == g);
+                if (has_eos) {  // rare: one group in the whole vocabulary
+                    if (full)
+                        walk_task<TabT, OutT, HAS_OUT, true, true>(p, first, tile, Cs, q0, nq, g, lane);
+                    else
+                        walk_task<TabT, OutT, HAS_OUT, false, true>(p, first, gtab, Cs, q0, nq, g, lane);
+                } else if (full) {
+                    walk_task<TabT, OutT, HAS_OUT, true, false>(p, first, tile, Cs, q0, nq, g, lane);
+                } else {
+                    walk_task<TabT, OutT, HAS_OUT, false, false>(p, first, gtab, Cs, q0, nq, g, lane);
+                }
             }
         }
     }
@@ -595,61 +624,40 @@ __device__ __forceinline__ void sparse_row(const WalkParams& p, const TabT* __re
         const int M = counts[1];
         int b = 0;
         for (int g0 = warp; g0 < M; g0 += kWalkWarps * kBatch) {
+            // issue the loads of kBatch chunks, then walk them one after the other
             uint4 rec[kBatch];
-            int32_t id[kBatch];
-            uint32_t st[kBatch];
-            bool cont[kBatch], act[kBatch];
+            int32_t id[kBatch];  // -1 = lane has no token in this chunk
+            uint32_t s1[kBatch];
 #pragma unroll
             for (int k = 0; k < kBatch; ++k) {
                 const int g = g0 + k * kWalkWarps;
                 rec[k] = make_uint4(0, 0, 0, 0);
-                id[k] = 0;
-                st[k] = dead;
-                act[k] = false;
+                id[k] = -1;
+                s1[k] = dead;
                 if (g < M) {
                     while (g >= cpre[b + 1]) ++b;
                     const LiveBucket lb = live[b];
                     const int i = (g - cpre[b]) * 32 + lane;
-                    st[k] = lb.s1;
+                    s1[k] = lb.s1;
                     if (i < lb.count) {
-                        act[k] = true;
                         rec[k] = __ldg(p.srec + lb.start + i);
                         id[k] = __ldg(p.sid + lb.start + i);
                     }
                 }
             }
-            bool any_cont = false;
 #pragma unroll
             for (int k = 0; k < kBatch; ++k) {
-                cont[k] = (rec[k].x & 0xFFu) > 1;
-                any_cont |= cont[k];
-            }
-            if (__any_sync(kFullWarp, any_cont)) {
-#pragma unroll
-                for (int j = 1; j < kInlineBytes; ++j) {
-                    any_cont = false;
-#pragma unroll
-                    for (int k = 0; k < kBatch; ++k) {
-                        if (cont[k]) {
-                            st[k] = lookup(st[k], tok_byte(rec[k], j));
-                            cont[k] = (st[k] != dead) && (j + 1 < static_cast<int>(rec[k].x & 0xFFu));
-                        }
-                        any_cont |= cont[k];
-                    }
-                    if (!__any_sync(kFullWarp, any_cont)) break;
-                }
-#pragma unroll
-                for (int k = 0; k < kBatch; ++k)
-                    if (cont[k])  // longer than the inline record: finish on the raw bytes
-                        st[k] = raw_walk(p, st[k], p.vocab_offsets[id[k]], p.vocab_offsets[id[k] + 1],
-                                         kInlineBytes);
-            }
-#pragma unroll
-            for (int k = 0; k < kBatch; ++k)
-                if (act[k] && st[k] != dead) {
-                    if (HAS_OUT) nrow[id[k]] = static_cast<OutT>(st[k]);
+                const int len = rec[k].x & 0xFFu;
+                bool go = len > 1;
+                uint32_t st = walk_rest<TabT, FULL>(tab, Cs, dead, rec[k], len, s1[k], go);
+                if (go)  // longer than the inline record: finish on the raw bytes
+                    st = raw_walk(p, st, p.vocab_offsets[id[k]], p.vocab_offsets[id[k] + 1],
+                                  kInlineBytes);
+                if (id[k] >= 0 && st != dead) {
+                    if (HAS_OUT) nrow[id[k]] = static_cast<OutT>(st);
                     atomicOr(&mrow[id[k] >> 5], 1u << (id[k] & 31));
                 }
+            }
         }
     } else if (q != p.dead) {
         for (int v = threadIdx.x; v < p.N; v += kWalkThreads) {
