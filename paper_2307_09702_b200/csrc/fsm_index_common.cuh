@@ -1,0 +1,200 @@
+// Shared definitions of the index-build kernels (paper Section 3, Algorithms 3 and 4).
+#pragma once
+
+#include "fsm_common.cuh"
+
+namespace fsm {
+namespace {
+
+constexpr int kHashBlocks = 64;
+constexpr int kMaxCs = 264;             // 256 classes + the null class, rounded up to 8
+constexpr int kWalkThreads = 1024;
+constexpr int kWalkWarps = kWalkThreads / 32;
+constexpr int kChunk = 32;              // states per warp task (dense walk)
+constexpr int kInlineBytes = 16;        // token bytes kept in a 16-byte record
+constexpr uint32_t kBulkChunk = 32768;  // bytes per bulk copy instruction (table staging)
+constexpr int kKeyStride = 129;         // second-level keys per first-byte class (two-level sort)
+constexpr int kKeys = kKeyStride * kKeyStride;
+constexpr int kTwoLevelMaxC = 127;      // more classes than this: one-level buckets only
+
+struct IndexMeta {
+    int32_t C;          // number of byte classes (the null class has id C)
+    int32_t Cs;         // row stride of the compressed table, entries
+    int32_t any_bad;    // set when the compressed table cannot be used (exact fallback)
+    int32_t two_level;  // tokens are bucketed by (class of byte 0, class of byte 1)
+};
+
+struct Workspace {
+    IndexMeta* meta;
+    uint8_t* cls;        // [256] byte -> class
+    uint8_t* class_rep;  // [256] class -> representative byte
+    uint64_t* partial;   // [kHashBlocks][256] column hash partial sums
+    void* table;         // [Q][Cs] of TabT
+    // dense walk: token records in token order (aliases the sparse walk's arrays)
+    uint4* tok_cls;      // [G*32] first 16 class ids of each token
+    uint8_t* tok_len;    // [G*32] min(length, 17)
+    // sparse walk: tokens sorted by bucket key
+    uint4* srec;         // [N] {min(len,17), class of byte 1..15}
+    int32_t* sid;        // [N] token id, same order as srec
+    int32_t* gcount;     // [256] tokens per first-byte class
+    int32_t* gstart;     // [257] first sorted position of each first-byte class
+    int32_t* count2;     // [kKeys] tokens per (first class, second key)
+    int32_t* cursor2;    // [kKeys] placement cursors
+    int32_t* start2;     // [kKeys] first sorted position of each (first class, second key)
+    size_t bytes;
+};
+
+inline size_t table_elem_bytes(int32_t Q) { return Q <= 65535 ? 2 : 4; }
+
+inline Workspace carve(void* base, int32_t Q, int32_t N) {
+    Workspace w;
+    uint8_t* p = static_cast<uint8_t*>(base);
+    size_t off = 0;
+    auto take = [&](size_t n) {
+        uint8_t* r = p ? p + off : nullptr;
+        off += align_up(n, 256);
+        return r;
+    };
+    const size_t G32 = (static_cast<size_t>(N) + 31) / 32 * 32;
+    w.meta = reinterpret_cast<IndexMeta*>(take(sizeof(IndexMeta)));
+    w.cls = take(256);
+    w.class_rep = take(256);
+    w.partial = reinterpret_cast<uint64_t*>(take(sizeof(uint64_t) * kHashBlocks * 256));
+    w.table = take(static_cast<size_t>(Q) * kMaxCs * table_elem_bytes(Q));
+    const size_t dense_bytes = G32 * sizeof(uint4) + G32;
+    const size_t srec_bytes = align_up(static_cast<size_t>(N) * sizeof(uint4), 256);
+    const size_t sparse_bytes = srec_bytes + static_cast<size_t>(N) * sizeof(int32_t);
+    uint8_t* tokens = take(dense_bytes > sparse_bytes ? dense_bytes : sparse_bytes);
+    w.tok_cls = reinterpret_cast<uint4*>(tokens);
+    w.tok_len = tokens ? tokens + G32 * sizeof(uint4) : nullptr;
+    w.srec = reinterpret_cast<uint4*>(tokens);
+    w.sid = reinterpret_cast<int32_t*>(tokens ? tokens + srec_bytes : nullptr);
+    w.gcount = reinterpret_cast<int32_t*>(take(256 * sizeof(int32_t)));
+    w.gstart = reinterpret_cast<int32_t*>(take(257 * sizeof(int32_t)));
+    w.count2 = reinterpret_cast<int32_t*>(take(kKeys * sizeof(int32_t)));
+    w.cursor2 = reinterpret_cast<int32_t*>(take(kKeys * sizeof(int32_t)));
+    w.start2 = reinterpret_cast<int32_t*>(take(kKeys * sizeof(int32_t)));
+    w.bytes = off;
+    return w;
+}
+
+struct WalkParams {
+    const void* table;
+    const IndexMeta* meta;
+    const int32_t* trans;
+    const uint8_t* accept;
+    const uint8_t* vocab_bytes;
+    const int32_t* vocab_offsets;
+    int64_t vocab_nbytes;
+    int32_t Q, N, G, dead, eos_id, q_begin, q_end;
+    uint32_t smem_cap;  // bytes of dynamic shared memory requested at launch
+    // dense walk
+    const uint4* tok_cls;
+    const uint8_t* tok_len;
+    // sparse walk
+    const uint4* srec;
+    const int32_t* sid;
+    const int32_t* gstart;
+    const int32_t* count2;
+    const int32_t* start2;
+    // outputs
+    uint32_t* mask;
+    void* next;
+    int32_t* status;
+};
+
+#ifdef __CUDACC__
+__device__ __forceinline__ uint64_t mix64(uint64_t x) {
+    x += 0x9E3779B97F4A7C15ull;
+    x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+    x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+    return x ^ (x >> 31);
+}
+
+__device__ __forceinline__ uint32_t clamp_state(int32_t v, int32_t Q, int32_t dead) {
+    return (static_cast<uint32_t>(v) >= static_cast<uint32_t>(Q)) ? dead : v;
+}
+
+// Bucket key of a token in the sorted order of the sparse walk.
+__device__ __forceinline__ int bucket_key(bool two_level, int first, int second_key) {
+    return two_level ? first * kKeyStride + second_key : first;
+}
+
+// Bounds-checked view of one token for the token-side preparation kernels.
+struct TokenInfo {
+    int64_t start;
+    int len;         // min(length, kInlineBytes + 1); 0 = not bucketed (empty, EOS, bad offsets)
+    int first;       // class of byte 0
+    int second_key;  // 0 for one-byte tokens, else 1 + class of byte 1
+};
+
+__device__ __forceinline__ TokenInfo token_info(const uint8_t* __restrict__ vocab_bytes,
+                                                const int32_t* __restrict__ vocab_offsets,
+                                                int64_t vocab_nbytes, int32_t N, int32_t eos_id,
+                                                const uint8_t* s_cls, int64_t v, bool* bad) {
+    TokenInfo t = {0, 0, 0, 0};
+    if (v < N && v != eos_id) {
+        const int64_t o0 = vocab_offsets[v], o1 = vocab_offsets[v + 1];
+        if (o0 < 0 || o1 < o0 || o1 > vocab_nbytes) {
+            *bad = true;
+        } else if (o1 > o0) {
+            t.start = o0;
+            t.len = static_cast<int>(min(o1 - o0, static_cast<int64_t>(kInlineBytes + 1)));
+            t.first = s_cls[vocab_bytes[o0]];
+            if (t.len > 1) t.second_key = 1 + s_cls[vocab_bytes[o0 + 1]];
+        }
+    }
+    return t;
+}
+
+__device__ __forceinline__ uint32_t tok_byte(const uint4& t, int i) {
+    const uint32_t w = (i >> 2) == 0 ? t.x : (i >> 2) == 1 ? t.y : (i >> 2) == 2 ? t.z : t.w;
+    return (w >> ((i & 3) * 8)) & 0xFFu;
+}
+
+// Walks bytes [from, o1 - o0) of a token through the uncompressed table.
+__device__ __noinline__ uint32_t raw_walk_impl(const int32_t* __restrict__ trans,
+                                               const uint8_t* __restrict__ vocab_bytes, int32_t Q,
+                                               int32_t dead, uint32_t s, int64_t o0, int64_t o1,
+                                               int from) {
+    for (int64_t i = o0 + from; i < o1 && s != static_cast<uint32_t>(dead); ++i)
+        s = clamp_state(trans[static_cast<size_t>(s) * 256 + vocab_bytes[i]], Q, dead);
+    return s;
+}
+
+__device__ __forceinline__ uint32_t raw_walk(const WalkParams& p, uint32_t s, int64_t o0,
+                                             int64_t o1, int from) {
+    return raw_walk_impl(p.trans, p.vocab_bytes, p.Q, p.dead, s, o0, o1, from);
+}
+
+// Bytes START.. of one token walked from state s, all 32 lanes in lock step.  `go`
+// says whether this lane still has a live walk with bytes left.  The loop is
+// warp-uniform (one vote per byte) and its body has no branches: lanes that are done
+// keep their state through a select.  Every state value is a valid table row
+// (out-of-range entries were replaced by `dead` when the table was compressed), so the
+// shared-memory lookup needs no guard; the global-memory lookup is predicated to save
+// traffic.  On return `go` is true only for tokens longer than the inline record.
+template <typename TabT, bool FULL, int START>
+__device__ __forceinline__ uint32_t walk_rest(const TabT* __restrict__ tab, uint32_t Cs,
+                                              uint32_t dead, const uint4& tk, int len, uint32_t s,
+                                              bool& go) {
+#pragma unroll
+    for (int i = START; i < kInlineBytes; ++i) {
+        if (!__any_sync(kFullWarp, go)) break;
+        const uint32_t c = tok_byte(tk, i);
+        uint32_t ns;
+        if (FULL) {
+            ns = tab[s * Cs + c];
+        } else {
+            ns = s;
+            if (go) ns = __ldg(tab + static_cast<size_t>(s) * Cs + c);
+        }
+        s = go ? ns : s;
+        go = go && (ns != dead) && (i + 1 < len);
+    }
+    return s;
+}
+#endif  // __CUDACC__
+
+}  // namespace
+}  // namespace fsm
