@@ -22,13 +22,14 @@ extern "C" size_t fsm_index_workspace_bytes(int32_t Q, int32_t N, int64_t vocab_
     return fsm::carve(nullptr, Q, N).bytes;
 }
 
-extern "C" int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* accept,
-                                    const uint8_t* vocab_bytes, const int32_t* vocab_offsets,
-                                    int64_t vocab_nbytes, int32_t Q, int32_t N,
-                                    int32_t dead_state, int32_t eos_id, int32_t q_begin,
-                                    int32_t q_end, uint32_t* allowed_mask, void* next_state,
-                                    int32_t state_dtype, void* workspace, size_t workspace_bytes,
-                                    int32_t* status_word, void* cuda_stream) {
+namespace {
+// `dense_only`: the workspace holds only what the dense walk needs (no survivor scratch).
+int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8_t* vocab_bytes,
+                    const int32_t* vocab_offsets, int64_t vocab_nbytes, int32_t Q, int32_t N,
+                    int32_t dead_state, int32_t eos_id, int32_t q_begin, int32_t q_end,
+                    uint32_t* allowed_mask, void* next_state, int32_t state_dtype, void* workspace,
+                    size_t workspace_bytes, int32_t* status_word, void* cuda_stream,
+                    bool dense_only) {
     using namespace fsm;
     if (Q <= 0 || N <= 0 || vocab_nbytes < 0 || N > 0x7FFFFFE0) return FSM_ERR_SHAPE;
     if (!dfa_trans || !accept || !vocab_offsets || !allowed_mask) return FSM_ERR_NULL;
@@ -44,7 +45,8 @@ extern "C" int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* acc
         return FSM_ERR_ALIGN;
     if (next_state && misaligned(next_state, state_dtype == FSM_STATE_U16 ? 2 : 4))
         return FSM_ERR_ALIGN;
-    const size_t need = fsm_index_workspace_bytes(Q, N, vocab_nbytes);
+    const Workspace sizes = carve(nullptr, Q, N);
+    const size_t need = dense_only ? sizes.dense_bytes : sizes.bytes;
     if (!workspace || workspace_bytes < need) return FSM_ERR_WORKSPACE;
     if (misaligned(workspace, 256)) return FSM_ERR_ALIGN;
     if (q_begin == q_end) return FSM_OK;
@@ -56,8 +58,13 @@ extern "C" int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* acc
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     Workspace ws = carve(workspace, Q, N);
     const bool wide = Q > 65535;
-    const bool sparse = tune.walk_algo != 1;
     const int G = (N + 31) / 32;
+    int cap = dev.smem_optin - 2048;  // static shared memory and alignment slack
+    if (tune.smem_table_cap > 0 && tune.smem_table_cap < cap) cap = tune.smem_table_cap;
+    // The sparse walk needs the survivor scratch and room for its per-warp staging.
+    const bool sparse = tune.walk_algo != 1 && !dense_only &&
+                        (N + kSlice - 1) / kSlice <= kMaxSlices &&
+                        sparse_fixed_smem<int32_t, true>(N) + 4096 <= static_cast<size_t>(dev.smem_optin - 2048);
 
     const int hash_blocks = Q < kHashBlocks ? Q : kHashBlocks;
     hash_columns<<<hash_blocks, 256, 0, stream>>>(dfa_trans, Q, dead_state, ws.partial,
@@ -110,9 +117,8 @@ extern "C" int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* acc
     p.mask = allowed_mask;
     p.next = next_state;
     p.status = status_word;
-    int cap = dev.smem_optin - 2048;  // static shared memory and alignment slack
-    if (tune.smem_table_cap > 0 && tune.smem_table_cap < cap) cap = tune.smem_table_cap;
-    const int min_cap = sparse ? static_cast<int>(kSparseFixedSmem) + 1024 : kChunk * kMaxCs * 4;
+    const int min_cap = sparse ? static_cast<int>(sparse_fixed_smem<int32_t, true>(N)) + 4096
+                               : kChunk * kMaxCs * 4;
     if (cap < min_cap) cap = min_cap;
     p.smem_cap = static_cast<uint32_t>(cap) / 128 * 128;
 
@@ -124,13 +130,14 @@ extern "C" int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* acc
         grid = (tasks + kWalkWarps - 1) / kWalkWarps;
     }
     if (grid > dev.sm_count) grid = dev.sm_count;
+    if (sparse && grid > kMaxSparseCtas) grid = kMaxSparseCtas;
     if (tune.walk_ctas > 0 && tune.walk_ctas < grid) grid = tune.walk_ctas;
     const int prof = profile_begin(stream);
     cudaError_t e;
     if (sparse)
-        e = wide ? launch_sparse_for<int32_t>(p, static_cast<int>(grid), state_dtype,
+        e = wide ? launch_sparse_for<int32_t>(p, ws.survivors, static_cast<int>(grid), state_dtype,
                                               next_state != nullptr, stream)
-                 : launch_sparse_for<uint16_t>(p, static_cast<int>(grid), state_dtype,
+                 : launch_sparse_for<uint16_t>(p, ws.survivors, static_cast<int>(grid), state_dtype,
                                                next_state != nullptr, stream);
     else
         e = wide ? launch_walk_for<int32_t>(p, static_cast<int>(grid), state_dtype,
@@ -139,6 +146,19 @@ extern "C" int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* acc
                                              next_state != nullptr, stream);
     profile_end(prof, stream);
     return e == cudaSuccess ? FSM_OK : FSM_ERR_CUDA;
+}
+}  // namespace
+
+extern "C" int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* accept,
+                                    const uint8_t* vocab_bytes, const int32_t* vocab_offsets,
+                                    int64_t vocab_nbytes, int32_t Q, int32_t N,
+                                    int32_t dead_state, int32_t eos_id, int32_t q_begin,
+                                    int32_t q_end, uint32_t* allowed_mask, void* next_state,
+                                    int32_t state_dtype, void* workspace, size_t workspace_bytes,
+                                    int32_t* status_word, void* cuda_stream) {
+    return build_rows_impl(dfa_trans, accept, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N,
+                           dead_state, eos_id, q_begin, q_end, allowed_mask, next_state,
+                           state_dtype, workspace, workspace_bytes, status_word, cuda_stream, false);
 }
 
 extern "C" int fsm_index_build(const int32_t* dfa_trans, const uint8_t* accept,
@@ -190,14 +210,15 @@ extern "C" int fsm_index_build_static(const int32_t* dfa_trans, const uint8_t* a
                                       void* next_state, int32_t state_dtype, int32_t* status_word,
                                       void* cuda_stream) {
     if (Q <= 0 || N <= 0 || vocab_nbytes < 0) return FSM_ERR_SHAPE;
-    const size_t need = fsm_index_workspace_bytes(Q, N, vocab_nbytes);
-    if (need == 0 || need > FSM_STATIC_SCRATCH_BYTES) return FSM_ERR_WORKSPACE;
+    // The built-in array is sized for the dense walk's scratch (no survivor lists).
+    const size_t need = fsm::carve(nullptr, Q, N).dense_bytes;
+    if (need > FSM_STATIC_SCRATCH_BYTES) return FSM_ERR_WORKSPACE;
     if (!fsm::device_info().ok) return FSM_ERR_CUDA;
     void* scratch = fsm::static_scratch_address();
     if (scratch == nullptr) return FSM_ERR_CUDA;
     // Every part of the scratch that the build reads is written earlier in the same build,
     // so the previous call's leftovers need no clearing.
-    return fsm_index_build_rows(dfa_trans, accept, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N,
-                                dead_state, eos_id, 0, Q, allowed_mask, next_state, state_dtype,
-                                scratch, FSM_STATIC_SCRATCH_BYTES, status_word, cuda_stream);
+    return build_rows_impl(dfa_trans, accept, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N,
+                           dead_state, eos_id, 0, Q, allowed_mask, next_state, state_dtype, scratch,
+                           FSM_STATIC_SCRATCH_BYTES, status_word, cuda_stream, true);
 }

@@ -16,6 +16,7 @@ constexpr uint32_t kBulkChunk = 32768;  // bytes per bulk copy instruction (tabl
 constexpr int kKeyStride = 129;         // second-level keys per first-byte class (two-level sort)
 constexpr int kKeys = kKeyStride * kKeyStride;
 constexpr int kTwoLevelMaxC = 127;      // more classes than this: one-level buckets only
+constexpr int kMaxSparseCtas = 160;     // CTAs of the sparse walk (one survivor scratch each)
 
 struct IndexMeta {
     int32_t C;          // number of byte classes (the null class has id C)
@@ -41,7 +42,9 @@ struct Workspace {
     int32_t* count2;     // [kKeys] tokens per (first class, second key)
     int32_t* cursor2;    // [kKeys] placement cursors
     int32_t* start2;     // [kKeys] first sorted position of each (first class, second key)
-    size_t bytes;
+    void* survivors;     // [kMaxSparseCtas][slices][256] survivor lists of the sparse walk
+    size_t bytes;        // everything above
+    size_t dense_bytes;  // without `survivors`: enough for the dense walk
 };
 
 inline size_t table_elem_bytes(int32_t Q) { return Q <= 65535 ? 2 : 4; }
@@ -74,6 +77,10 @@ inline Workspace carve(void* base, int32_t Q, int32_t N) {
     w.count2 = reinterpret_cast<int32_t*>(take(kKeys * sizeof(int32_t)));
     w.cursor2 = reinterpret_cast<int32_t*>(take(kKeys * sizeof(int32_t)));
     w.start2 = reinterpret_cast<int32_t*>(take(kKeys * sizeof(int32_t)));
+    w.dense_bytes = off;
+    const size_t ctas = Q < kMaxSparseCtas ? Q : kMaxSparseCtas;
+    const size_t slice_slots = (static_cast<size_t>(N) + 255) / 256 * 256;
+    w.survivors = take(ctas * slice_slots * (Q <= 65535 ? 4 : 8));
     w.bytes = off;
     return w;
 }

@@ -2,25 +2,25 @@
 //
 // Most (state, token) walks die on their first or second byte.  Tokens are therefore
 // kept sorted by bucket key - the class of byte 0 and (with few enough classes) the class
-// of byte 1 - so that one table lookup settles a whole bucket:
+// of byte 1 - so that one table lookup settles a whole bucket.  One persistent CTA per
+// SM works on one index row (one state q) at a time; the compressed table is staged in
+// shared memory once (bulk async copy) when it fits, else lookups use the read-only cache.
 //
-//   fill    every row of the next-state table is first set to `dead` and its bitmask
-//           row to 0.  The fill is done by the bulk-copy engine (cp.async.bulk, shared
-//           -> global) from a constant buffer in shared memory, issued one row ahead of
-//           the walk by a single thread, so it costs no issue slots and overlaps the
-//           walk of the previous row.
-//   walk    for a state q, only buckets whose key q can read are visited: a unit of
-//           work is (readable first class, block of 32 second keys); the units of all
-//           rows of a CTA are dealt round-robin to its 32 warps, which work without any
-//           CTA-wide barrier.  Inside a bucket, lane = token, 32 tokens at a time, from
-//           the first byte the bucket key does not cover.
-//   scatter survivors store their end state into the row and OR their bit into the
-//           bitmask row.  The row was written moments earlier from the same SM, so these
-//           partial writes merge in L2.
+//   walk      only buckets whose key q can read are visited.  A unit of work is
+//             (readable first class, block of 32 second keys); warps take units from a
+//             shared counter.  Inside a bucket, lane = token, 32 tokens at a time,
+//             starting at the first byte the bucket key does not cover.  A surviving
+//             token appends (id within slice, end state) to the list of its *slice*
+//             (kSlice consecutive token ids).  The lists live in a per-CTA scratch in
+//             global memory that stays L2 resident; a list can hold a whole slice, so
+//             nothing can overflow.
+//   assemble  each warp takes slices in turn: it fills a 1 KB staging buffer in shared
+//             memory with `dead`, writes the slice's survivors into it, and stores the
+//             finished slice of the next-state row and its bitmask words with coalesced
+//             16-byte stores.  Global memory only sees full, write-once traffic for the
+//             outputs: the tokens whose first byte q cannot read cost no lookup at all.
 //
-// One persistent CTA per SM; the compressed table is staged in shared memory once
-// (bulk async copy) when it fits, else lookups go through the read-only cache.
-// Results are identical to the dense walk.
+// Three CTA barriers per row.  Results are identical to the dense walk.
 #pragma once
 
 #include "fsm_index_common.cuh"
@@ -28,61 +28,39 @@
 namespace fsm {
 namespace {
 
-constexpr uint32_t kFillBytes = 16384;  // shared-memory source of the row fill
-constexpr uint32_t kZeroBytes = 4096;   // shared-memory source of the bitmask fill
-constexpr uint32_t kSparseFixedSmem = kFillBytes + kZeroBytes;
+constexpr int kSliceShift = 8;
+constexpr int kSlice = 1 << kSliceShift;  // token ids per assembly slice
+constexpr int kSliceWords = kSlice / 32;
+constexpr int kMaxSlices = 8192;          // vocabularies up to 2 M tokens (else the dense walk)
 
-__device__ __forceinline__ void bulk_store_s2g(void* dst, const void* src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst),
-                 "r"(smem_addr(src)), "r"(bytes)
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_commit() {
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-template <int kPending>
-__device__ __forceinline__ void bulk_wait() {
-    asm volatile("cp.async.bulk.wait_group %0;" ::"n"(kPending) : "memory");
-}
-__device__ __forceinline__ void fence_proxy_async() {
-    asm volatile("fence.proxy.async;" ::: "memory");
-}
+// Survivor record: token id within its slice and end state.
+template <typename TabT> struct Entry;
+template <> struct Entry<uint16_t> {
+    using type = uint32_t;
+    __device__ static type pack(uint32_t lid, uint32_t s) { return (s << 16) | lid; }
+    __device__ static uint32_t lid(type e) { return e & 0xFFFFu; }
+    __device__ static uint32_t state(type e) { return e >> 16; }
+};
+template <> struct Entry<int32_t> {
+    using type = unsigned long long;
+    __device__ static type pack(uint32_t lid, uint32_t s) { return (static_cast<type>(s) << 32) | lid; }
+    __device__ static uint32_t lid(type e) { return static_cast<uint32_t>(e); }
+    __device__ static uint32_t state(type e) { return static_cast<uint32_t>(e >> 32); }
+};
 
-// Fills `count` elements at `dst` with the pattern held in `src` (a shared-memory
-// buffer of `src_bytes` bytes): the 16-byte aligned middle by bulk stores, the ragged
-// head and tail with plain stores.  Called by one thread.
-template <typename T>
-__device__ __forceinline__ void fill_async(T* dst, int64_t count, T value, const void* src,
-                                           uint32_t src_bytes) {
-    const uintptr_t addr = reinterpret_cast<uintptr_t>(dst);
-    int64_t head = static_cast<int64_t>(((16 - (addr & 15)) & 15) / sizeof(T));
-    if (head > count) head = count;
-    for (int64_t i = 0; i < head; ++i) dst[i] = value;
-    const int64_t mid_bytes = (count - head) * static_cast<int64_t>(sizeof(T)) / 16 * 16;
-    uint8_t* mid = reinterpret_cast<uint8_t*>(dst + head);
-    for (int64_t o = 0; o < mid_bytes; o += src_bytes) {
-        const int64_t left = mid_bytes - o;
-        bulk_store_s2g(mid + o, src, left < src_bytes ? static_cast<uint32_t>(left) : src_bytes);
-    }
-    for (int64_t i = head + mid_bytes / static_cast<int64_t>(sizeof(T)); i < count; ++i) dst[i] = value;
-}
-
-// Bounded wait for the fill of this CTA's k-th row.
-__device__ __forceinline__ bool wait_row_filled(const int* flag, int k) {
-    for (uint32_t it = 0; it < (1u << 22); ++it) {
-        int v;
-        asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(v) : "r"(smem_addr(flag)) : "memory");
-        if (v >= k) return true;
-        __nanosleep(64);
-    }
-    return false;
-}
+// Where the survivors of the row being walked go.
+template <typename TabT>
+struct SurvivorSink {
+    typename Entry<TabT>::type* lists;  // [nslices][kSlice], this CTA's part of the scratch
+    int* counts;                        // [nslices], shared memory
+    int* unit_ctr;                      // shared memory
+};
 
 // One chunk: up to 32 tokens of a bucket (lane = token), starting at sorted position
 // `pos`, all in state `s` after the DEPTH bytes the bucket key covers.
-template <typename TabT, typename OutT, bool HAS_OUT, bool FULL, int DEPTH>
+template <typename TabT, bool FULL, int DEPTH>
 __device__ __forceinline__ void walk_chunk(const WalkParams& p, const TabT* __restrict__ tab,
-                                           uint32_t Cs, OutT* nrow, uint32_t* mrow, int pos,
+                                           uint32_t Cs, const SurvivorSink<TabT>& sink, int pos,
                                            int count, uint32_t s, int lane) {
     const uint32_t dead = p.dead;
     uint4 rec = make_uint4(0, 0, 0, 0);
@@ -97,125 +75,146 @@ __device__ __forceinline__ void walk_chunk(const WalkParams& p, const TabT* __re
     if (go)  // longer than the inline record and still alive: finish on the raw bytes
         st = raw_walk(p, st, p.vocab_offsets[id], p.vocab_offsets[id + 1], kInlineBytes);
     if (id >= 0 && st != dead) {
-        if (HAS_OUT) nrow[id] = static_cast<OutT>(st);
-        atomicOr(&mrow[id >> 5], 1u << (id & 31));
+        const int slice = id >> kSliceShift;
+        const int at = atomicAdd(&sink.counts[slice], 1);  // < kSlice: a token survives once
+        sink.lists[static_cast<size_t>(slice) * kSlice + at] =
+            Entry<TabT>::pack(id & (kSlice - 1), st);
     }
 }
 
-template <typename TabT, typename OutT, bool HAS_OUT, bool FULL>
-__device__ __forceinline__ void sparse_rows(const WalkParams& p, const TabT* __restrict__ tab,
-                                            int C, uint32_t Cs, bool two_level,
-                                            const int32_t* s_gstart, int* filled,
-                                            const void* fillbuf, const void* zerobuf, int nmine) {
+// Walks every readable bucket of state q; warps take units from sink.unit_ctr.
+template <typename TabT, bool FULL>
+__device__ __forceinline__ void walk_row(const WalkParams& p, const TabT* __restrict__ tab, int C,
+                                         uint32_t Cs, bool two_level, const int32_t* s_gstart,
+                                         const SurvivorSink<TabT>& sink, int q) {
     const uint32_t dead = p.dead;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
     auto lookup = [&](uint32_t s, uint32_t c) -> uint32_t {
         if (FULL) return tab[s * Cs + c];
         return __ldg(tab + static_cast<size_t>(s) * Cs + c);
     };
-    auto issue_fill = [&](int k) {  // thread 0 only
-        const int r = blockIdx.x + k * gridDim.x;
-        if (HAS_OUT)
-            fill_async<OutT>(static_cast<OutT*>(p.next) + static_cast<size_t>(r) * p.N, p.N,
-                             static_cast<OutT>(dead), fillbuf, kFillBytes);
-        fill_async<uint32_t>(p.mask + static_cast<size_t>(r) * p.G, p.G, 0u, zerobuf, kZeroBytes);
-        bulk_commit();
-    };
-
-    if (threadIdx.x == 0 && nmine > 0) issue_fill(0);
-    const int KB = two_level ? (C + 1 + 31) / 32 : 1;  // blocks of 32 second-level keys
-    int u_base = 0;                                    // units dealt so far, modulo 32
-    for (int k = 0; k < nmine; ++k) {
-        const int r = blockIdx.x + k * gridDim.x;
-        const int q = p.q_begin + r;
-        if (threadIdx.x == 0) {
-            // keep the fill one row ahead, then publish that row k is ready
-            if (k + 1 < nmine) {
-                issue_fill(k + 1);
-                bulk_wait<1>();
-            } else {
-                bulk_wait<0>();
-            }
-            fence_proxy_async();
-            asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_addr(filled)), "r"(k) : "memory");
+    // readable, non-empty first-byte classes of state q
+    uint32_t lm[8];
+    int n_live = 0;
+#pragma unroll
+    for (int cb = 0; cb < 8; ++cb) {
+        lm[cb] = 0;
+        if (cb * 32 < C) {
+            const int c = cb * 32 + lane;
+            bool ok = false;
+            if (c < C) ok = (lookup(q, c) != dead) && (s_gstart[c + 1] > s_gstart[c]);
+            lm[cb] = __ballot_sync(kFullWarp, ok);
+            n_live += __popc(lm[cb]);
         }
-        __syncwarp();
-        // readable, non-empty first-byte classes of state q
-        uint32_t lm[8];
-        int n_live = 0;
+    }
+    const int KB = two_level ? (C + 1 + 31) / 32 : 1;  // blocks of 32 second-level keys
+    const int U = n_live * KB;
+    while (true) {
+        int j = 0;
+        if (lane == 0) j = atomicAdd(sink.unit_ctr, 1);
+        j = __shfl_sync(kFullWarp, j, 0);
+        if (j >= U) break;
+        const int li = j / KB, kb = j - li * KB;
+        int c0 = 0, rem = li;  // the li-th readable class
 #pragma unroll
         for (int cb = 0; cb < 8; ++cb) {
-            lm[cb] = 0;
-            if (cb * 32 < C) {
-                const int c = cb * 32 + lane;
-                bool ok = false;
-                if (c < C) ok = (lookup(q, c) != dead) && (s_gstart[c + 1] > s_gstart[c]);
-                lm[cb] = __ballot_sync(kFullWarp, ok);
-                n_live += __popc(lm[cb]);
+            const int pc = __popc(lm[cb]);
+            if (rem >= 0 && rem < pc) {
+                c0 = cb * 32 + __fns(lm[cb], 0, rem + 1);
+                rem = -1;
+            } else if (rem >= 0) {
+                rem -= pc;
             }
         }
-        const int U = n_live * KB;
-        const int first = (warp - u_base) & 31;
-        u_base = (u_base + U) & 31;
-        const bool eos_mine = (p.eos_id >= 0) && ((k & 31) == warp);
-        if (first >= U && !eos_mine) continue;
-        if (!wait_row_filled(filled, k)) {
-            if (lane == 0) raise_flag(p.status, FSM_FLAG_WAIT_TIMEOUT);
-            return;
+        const uint32_t s1 = lookup(q, c0);
+        // lane = second-level key: bucket size, position and state after its bytes
+        int cnt = 0, start = 0;
+        uint32_t s2 = dead;
+        if (two_level) {
+            const int key2 = kb * 32 + lane;
+            if (key2 <= C) {
+                cnt = __ldg(p.count2 + c0 * kKeyStride + key2);
+                start = __ldg(p.start2 + c0 * kKeyStride + key2);
+                s2 = (key2 == 0) ? s1 : lookup(s1, key2 - 1);
+            }
+        } else if (lane == 0) {
+            start = s_gstart[c0];
+            cnt = s_gstart[c0 + 1] - start;
+            s2 = s1;
         }
-        OutT* nrow = HAS_OUT ? static_cast<OutT*>(p.next) + static_cast<size_t>(r) * p.N : nullptr;
-        uint32_t* mrow = p.mask + static_cast<size_t>(r) * p.G;
-        if (eos_mine && lane == 0 && q != p.dead && p.accept[q]) {
-            if (HAS_OUT) nrow[p.eos_id] = static_cast<OutT>(q);
-            atomicOr(&mrow[p.eos_id >> 5], 1u << (p.eos_id & 31));
+        uint32_t m = __ballot_sync(kFullWarp, cnt > 0 && s2 != dead);
+        while (m) {
+            const int l = __ffs(m) - 1;
+            m &= m - 1;
+            const int bstart = __shfl_sync(kFullWarp, start, l);
+            const int bn = __shfl_sync(kFullWarp, cnt, l);
+            const uint32_t bs = __shfl_sync(kFullWarp, s2, l);
+            if (two_level && !(kb == 0 && l == 0)) {
+                for (int i0 = 0; i0 < bn; i0 += 32)
+                    walk_chunk<TabT, FULL, 2>(p, tab, Cs, sink, bstart + i0, bn - i0, bs, lane);
+            } else {
+                for (int i0 = 0; i0 < bn; i0 += 32)
+                    walk_chunk<TabT, FULL, 1>(p, tab, Cs, sink, bstart + i0, bn - i0, bs, lane);
+            }
         }
-        for (int j = first; j < U; j += 32) {
-            const int li = j / KB, kb = j - li * KB;
-            int c0 = 0, rem = li;  // the li-th readable class
+    }
+}
+
+// Assembles and stores the slices of one row; warp w takes slices w, w+32, ...
+template <typename TabT, typename OutT, bool HAS_OUT>
+__device__ __forceinline__ void assemble_row(const WalkParams& p, const SurvivorSink<TabT>& sink,
+                                             OutT* stage, uint32_t* mwords, int nslices, int q,
+                                             OutT* nrow, uint32_t* mrow) {
+    using E = Entry<TabT>;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t dead = p.dead;
+    const uint32_t d32 = sizeof(OutT) == 2 ? (dead | (dead << 16)) : dead;
+    const uint4 dead16 = make_uint4(d32, d32, d32, d32);
+    constexpr int kVec = 16 / sizeof(OutT);          // elements per 16-byte vector
+    constexpr int kVecPerLane = kSlice / kVec / 32;  // 2 (int32) or 1 (uint16)
+    const bool eos_ok = p.eos_id >= 0 && q != p.dead && p.accept[q];
+    for (int sl = warp; sl < nslices; sl += kWalkWarps) {
+        const int base = sl << kSliceShift;
+        const int n = min(kSlice, p.N - base);
+        const int cnt = sink.counts[sl];
+        // the first 32 survivors are fetched before the fill to overlap their latency
+        typename E::type e0 = 0;
+        if (lane < cnt) e0 = sink.lists[static_cast<size_t>(sl) * kSlice + lane];
+        if (HAS_OUT) {
 #pragma unroll
-            for (int cb = 0; cb < 8; ++cb) {
-                const int pc = __popc(lm[cb]);
-                if (rem >= 0 && rem < pc) {
-                    c0 = cb * 32 + __fns(lm[cb], 0, rem + 1);
-                    rem = -1;
-                } else if (rem >= 0) {
-                    rem -= pc;
-                }
-            }
-            const uint32_t s1 = lookup(q, c0);
-            // lane = second-level key: bucket size, position and state after its bytes
-            int cnt = 0, start = 0;
-            uint32_t s2 = dead;
-            if (two_level) {
-                const int key2 = kb * 32 + lane;
-                if (key2 <= C) {
-                    cnt = __ldg(p.count2 + c0 * kKeyStride + key2);
-                    start = __ldg(p.start2 + c0 * kKeyStride + key2);
-                    s2 = (key2 == 0) ? s1 : lookup(s1, key2 - 1);
-                }
-            } else if (lane == 0) {
-                start = s_gstart[c0];
-                cnt = s_gstart[c0 + 1] - start;
-                s2 = s1;
-            }
-            uint32_t m = __ballot_sync(kFullWarp, cnt > 0 && s2 != dead);
-            while (m) {
-                const int l = __ffs(m) - 1;
-                m &= m - 1;
-                const int bstart = __shfl_sync(kFullWarp, start, l);
-                const int bn = __shfl_sync(kFullWarp, cnt, l);
-                const uint32_t bs = __shfl_sync(kFullWarp, s2, l);
-                if (two_level && !(kb == 0 && l == 0)) {
-                    for (int i0 = 0; i0 < bn; i0 += 32)
-                        walk_chunk<TabT, OutT, HAS_OUT, FULL, 2>(p, tab, Cs, nrow, mrow, bstart + i0,
-                                                                 bn - i0, bs, lane);
-                } else {
-                    for (int i0 = 0; i0 < bn; i0 += 32)
-                        walk_chunk<TabT, OutT, HAS_OUT, FULL, 1>(p, tab, Cs, nrow, mrow, bstart + i0,
-                                                                 bn - i0, bs, lane);
-                }
+            for (int k = 0; k < kVecPerLane; ++k)
+                reinterpret_cast<uint4*>(stage)[lane + 32 * k] = dead16;
+        }
+        if (lane < kSliceWords) mwords[lane] = 0;
+        __syncwarp();
+        if (lane < cnt) {
+            if (HAS_OUT) stage[E::lid(e0)] = static_cast<OutT>(E::state(e0));
+            atomicOr(&mwords[E::lid(e0) >> 5], 1u << (E::lid(e0) & 31));
+        }
+        for (int i = 32 + lane; i < cnt; i += 32) {
+            const typename E::type e = sink.lists[static_cast<size_t>(sl) * kSlice + i];
+            if (HAS_OUT) stage[E::lid(e)] = static_cast<OutT>(E::state(e));
+            atomicOr(&mwords[E::lid(e) >> 5], 1u << (E::lid(e) & 31));
+        }
+        if (eos_ok && lane == 0 && p.eos_id >= base && p.eos_id < base + n) {
+            const int e = p.eos_id - base;
+            if (HAS_OUT) stage[e] = static_cast<OutT>(q);
+            atomicOr(&mwords[e >> 5], 1u << (e & 31));
+        }
+        __syncwarp();
+        if (lane < (n + 31) / 32) mrow[(base >> 5) + lane] = mwords[lane];
+        if (HAS_OUT) {
+            OutT* dst = nrow + base;
+            if (n == kSlice && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+#pragma unroll
+                for (int k = 0; k < kVecPerLane; ++k)
+                    reinterpret_cast<uint4*>(dst)[lane + 32 * k] =
+                        reinterpret_cast<const uint4*>(stage)[lane + 32 * k];
+            } else {  // ragged last slice or unaligned row: element-wise, still coalesced
+                for (int i = lane; i < n; i += 32) dst[i] = stage[i];
             }
         }
+        __syncwarp();  // staging is refilled by the next slice
     }
 }
 
@@ -253,42 +252,41 @@ __device__ void raw_rows(const WalkParams& p) {
 }
 
 template <typename TabT, typename OutT, bool HAS_OUT>
-__global__ void __launch_bounds__(kWalkThreads, 1) walk_sparse(const WalkParams p) {
+__global__ void __launch_bounds__(kWalkThreads, 1)
+walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t table_cap) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     __shared__ uint64_t bar;
-    __shared__ int filled;
     __shared__ int32_t s_gstart[260];
-    uint8_t* fillbuf = smem_raw;
-    uint8_t* zerobuf = smem_raw + kFillBytes;
-    TabT* stab = reinterpret_cast<TabT*>(smem_raw + kSparseFixedSmem);
+    __shared__ int s_unit_ctr;
 
     if (p.meta->any_bad != 0) {
         raw_rows<OutT, HAS_OUT>(p);
         return;
     }
+    const int nslices = (p.N + kSlice - 1) >> kSliceShift;
+    // dynamic shared memory: per-warp staging, per-warp bitmask words, slice counters, table
+    constexpr size_t kStageBytes = HAS_OUT ? kSlice * sizeof(OutT) : 0;
+    const int warp = threadIdx.x >> 5;
+    OutT* stage = reinterpret_cast<OutT*>(smem_raw + warp * kStageBytes);
+    uint32_t* mwords = reinterpret_cast<uint32_t*>(smem_raw + kWalkWarps * kStageBytes) + warp * kSliceWords;
+    int* counts = reinterpret_cast<int*>(smem_raw + kWalkWarps * (kStageBytes + kSliceWords * 4));
+    const size_t table_off = (kWalkWarps * (kStageBytes + kSliceWords * 4) +
+                              static_cast<size_t>(nslices) * 4 + 127) / 128 * 128;
+    TabT* stab = reinterpret_cast<TabT*>(smem_raw + table_off);
+
     const TabT* gtab = static_cast<const TabT*>(p.table);
-    const int C = p.meta->C, Cs = p.meta->Cs;
+    const int C = p.meta->C;
+    const uint32_t Cs = p.meta->Cs;
     const bool two_level = p.meta->two_level != 0;
     const uint64_t table_bytes = static_cast<uint64_t>(p.Q) * Cs * sizeof(TabT);
-    const bool full = p.smem_cap > kSparseFixedSmem && table_bytes <= p.smem_cap - kSparseFixedSmem;
-
-    // constant sources of the fills, bucket starts, table
-    {
-        const uint32_t d = sizeof(OutT) == 2 ? (p.dead | (p.dead << 16)) : p.dead;
-        for (uint32_t i = threadIdx.x; i < kFillBytes / 16; i += kWalkThreads)
-            reinterpret_cast<uint4*>(fillbuf)[i] = make_uint4(d, d, d, d);
-        for (uint32_t i = threadIdx.x; i < kZeroBytes / 16; i += kWalkThreads)
-            reinterpret_cast<uint4*>(zerobuf)[i] = make_uint4(0, 0, 0, 0);
-        for (int i = threadIdx.x; i < 257; i += kWalkThreads) s_gstart[i] = p.gstart[i];
+    const bool full = table_bytes <= table_cap;
+    for (int i = threadIdx.x; i < 257; i += kWalkThreads) s_gstart[i] = p.gstart[i];
+    if (full) {
         if (threadIdx.x == 0) {
-            filled = -1;
             mbar_init(&bar, 1);
             fence_mbar_init();
         }
-        fence_proxy_async();  // the bulk engine reads fillbuf / zerobuf written above
-    }
-    __syncthreads();
-    if (full) {
+        __syncthreads();
         if (threadIdx.x == 0) {
             const uint32_t bytes = static_cast<uint32_t>(table_bytes);
             mbar_expect_tx(&bar, bytes);
@@ -304,34 +302,57 @@ __global__ void __launch_bounds__(kWalkThreads, 1) walk_sparse(const WalkParams 
             return;
         }
     }
+    SurvivorSink<TabT> sink;
+    sink.lists = scratch + static_cast<size_t>(blockIdx.x) * nslices * kSlice;
+    sink.counts = counts;
+    sink.unit_ctr = &s_unit_ctr;
+
     const int nrows = p.q_end - p.q_begin;
-    const int nmine = nrows > static_cast<int>(blockIdx.x)
-                          ? (nrows - blockIdx.x + gridDim.x - 1) / gridDim.x
-                          : 0;
-    if (full)
-        sparse_rows<TabT, OutT, HAS_OUT, true>(p, stab, C, Cs, two_level, s_gstart, &filled, fillbuf,
-                                               zerobuf, nmine);
-    else
-        sparse_rows<TabT, OutT, HAS_OUT, false>(p, gtab, C, Cs, two_level, s_gstart, &filled, fillbuf,
-                                                zerobuf, nmine);
+    for (int r = blockIdx.x; r < nrows; r += gridDim.x) {
+        const int q = p.q_begin + r;
+        OutT* nrow = HAS_OUT ? static_cast<OutT*>(p.next) + static_cast<size_t>(r) * p.N : nullptr;
+        uint32_t* mrow = p.mask + static_cast<size_t>(r) * p.G;
+        for (int i = threadIdx.x; i < nslices; i += kWalkThreads) counts[i] = 0;
+        if (threadIdx.x == 0) s_unit_ctr = 0;
+        __syncthreads();
+        if (full)
+            walk_row<TabT, true>(p, stab, C, Cs, two_level, s_gstart, sink, q);
+        else
+            walk_row<TabT, false>(p, gtab, C, Cs, two_level, s_gstart, sink, q);
+        __syncthreads();  // every survivor of the row is in its list (stores visible CTA-wide)
+        assemble_row<TabT, OutT, HAS_OUT>(p, sink, stage, mwords, nslices, q, nrow, mrow);
+        __syncthreads();  // counters and lists are reused by the next row
+    }
+}
+
+// Shared-memory bytes of walk_sparse besides the table.
+template <typename OutT, bool HAS_OUT>
+size_t sparse_fixed_smem(int32_t N) {
+    const size_t nslices = (static_cast<size_t>(N) + kSlice - 1) >> kSliceShift;
+    const size_t stage = HAS_OUT ? kSlice * sizeof(OutT) : 0;
+    return (kWalkWarps * (stage + kSliceWords * 4) + nslices * 4 + 127) / 128 * 128;
 }
 
 template <typename TabT, typename OutT, bool HAS_OUT>
-cudaError_t launch_sparse(const WalkParams& p, int grid, cudaStream_t stream) {
+cudaError_t launch_sparse(const WalkParams& p, void* scratch, int grid, cudaStream_t stream) {
     auto kernel = walk_sparse<TabT, OutT, HAS_OUT>;
+    const size_t fixed = sparse_fixed_smem<OutT, HAS_OUT>(p.N);
+    if (fixed + 1024 > p.smem_cap) return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(p.smem_cap));
     if (e != cudaSuccess) return e;
-    kernel<<<grid, kWalkThreads, p.smem_cap, stream>>>(p);
+    kernel<<<grid, kWalkThreads, p.smem_cap, stream>>>(
+        p, static_cast<typename Entry<TabT>::type*>(scratch),
+        static_cast<uint32_t>(p.smem_cap - fixed));
     return cudaGetLastError();
 }
 
 template <typename TabT>
-cudaError_t launch_sparse_for(const WalkParams& p, int grid, int32_t state_dtype, bool has_out,
-                              cudaStream_t stream) {
-    if (!has_out) return launch_sparse<TabT, int32_t, false>(p, grid, stream);
-    if (state_dtype == FSM_STATE_U16) return launch_sparse<TabT, uint16_t, true>(p, grid, stream);
-    return launch_sparse<TabT, int32_t, true>(p, grid, stream);
+cudaError_t launch_sparse_for(const WalkParams& p, void* scratch, int grid, int32_t state_dtype,
+                              bool has_out, cudaStream_t stream) {
+    if (!has_out) return launch_sparse<TabT, int32_t, false>(p, scratch, grid, stream);
+    if (state_dtype == FSM_STATE_U16) return launch_sparse<TabT, uint16_t, true>(p, scratch, grid, stream);
+    return launch_sparse<TabT, int32_t, true>(p, scratch, grid, stream);
 }
 
 }  // namespace

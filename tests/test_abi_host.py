@@ -45,7 +45,7 @@ def test_workspace_query(fg):
     a = fg.fsm_index_workspace_bytes(1001, 128256, 505341)
     b = fg.fsm_index_workspace_bytes(20001, 152064, 601443)
     c = fg.fsm_index_workspace_bytes(70000, 152064, 601443)
-    assert 0 < a < b < c < 100 << 20 and a % 256 == 0
+    assert 0 < a < b < c < 512 << 20 and a % 256 == 0
 
 
 def test_index_build_rejects_bad_arguments_before_any_launch(fg):
