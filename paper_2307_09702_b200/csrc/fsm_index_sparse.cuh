@@ -32,6 +32,7 @@ constexpr int kSliceShift = 8;
 constexpr int kSlice = 1 << kSliceShift;  // token ids per assembly slice
 constexpr int kSliceWords = kSlice / 32;
 constexpr int kMaxSlices = 8192;          // vocabularies up to 2 M tokens (else the dense walk)
+constexpr int kDescCap = 4096;            // chunk descriptors kept per row
 
 // Survivor record: token id within its slice and end state.
 template <typename TabT> struct Entry;
@@ -48,27 +49,59 @@ template <> struct Entry<int32_t> {
     __device__ static uint32_t state(type e) { return static_cast<uint32_t>(e >> 32); }
 };
 
-// Where the survivors of the row being walked go.
+// Chunk descriptor: up to 32 tokens at sorted position `start`, all in `state` after
+// the `depth` bytes their bucket key covers.
+template <typename TabT> struct Desc;
+template <> struct Desc<uint16_t> {
+    using type = uint2;
+    __device__ static type pack(int start, uint32_t state, int count, int depth) {
+        return make_uint2(start, state | ((count - 1) << 16) | ((depth - 1) << 21));
+    }
+    __device__ static int start(type d) { return d.x; }
+    __device__ static uint32_t state(type d) { return d.y & 0xFFFFu; }
+    __device__ static int count(type d) { return ((d.y >> 16) & 31) + 1; }
+    __device__ static int depth(type d) { return ((d.y >> 21) & 1) + 1; }
+};
+template <> struct Desc<int32_t> {
+    using type = uint4;
+    __device__ static type pack(int start, uint32_t state, int count, int depth) {
+        return make_uint4(start, state, count, depth);
+    }
+    __device__ static int start(type d) { return d.x; }
+    __device__ static uint32_t state(type d) { return d.y; }
+    __device__ static int count(type d) { return d.z; }
+    __device__ static int depth(type d) { return d.w; }
+};
+
+// Shared state of the row being walked.
 template <typename TabT>
 struct SurvivorSink {
     typename Entry<TabT>::type* lists;  // [nslices][kSlice], this CTA's part of the scratch
     int* counts;                        // [nslices], shared memory
-    int* unit_ctr;                      // shared memory
+    typename Desc<TabT>::type* descs;   // [desc_cap] chunk descriptors, shared memory
+    int desc_cap;
+    int* ctrs;                          // shared: [0] unit counter, [1] descriptors written,
+                                        //         [2] chunk counter, [3] descriptor overflow
 };
 
-// One chunk: up to 32 tokens of a bucket (lane = token), starting at sorted position
-// `pos`, all in state `s` after the DEPTH bytes the bucket key covers.
-template <typename TabT, bool FULL, int DEPTH>
-__device__ __forceinline__ void walk_chunk(const WalkParams& p, const TabT* __restrict__ tab,
-                                           uint32_t Cs, const SurvivorSink<TabT>& sink, int pos,
-                                           int count, uint32_t s, int lane) {
-    const uint32_t dead = p.dead;
-    uint4 rec = make_uint4(0, 0, 0, 0);
-    int32_t id = -1;
+// One chunk: up to 32 tokens of a bucket (lane = token).  chunk_load fetches the lane's
+// record and token id; chunk_finish walks the rest of the token from state `s` (after
+// the DEPTH bytes the bucket key covers) and appends a survivor to its slice's list.
+__device__ __forceinline__ void chunk_load(const WalkParams& p, int pos, int count, int lane,
+                                           uint4& rec, int32_t& id) {
+    rec = make_uint4(0, 0, 0, 0);
+    id = -1;
     if (lane < count) {
         rec = __ldg(p.srec + pos + lane);
         id = __ldg(p.sid + pos + lane);
     }
+}
+
+template <typename TabT, bool FULL, int DEPTH>
+__device__ __forceinline__ void chunk_finish(const WalkParams& p, const TabT* __restrict__ tab,
+                                             uint32_t Cs, const SurvivorSink<TabT>& sink,
+                                             const uint4& rec, int32_t id, uint32_t s) {
+    const uint32_t dead = p.dead;
     const int len = rec.x & 0xFFu;
     bool go = len > DEPTH;
     uint32_t st = walk_rest<TabT, FULL, DEPTH>(tab, Cs, dead, rec, len, s, go);
@@ -82,8 +115,22 @@ __device__ __forceinline__ void walk_chunk(const WalkParams& p, const TabT* __re
     }
 }
 
-// Walks every readable bucket of state q; warps take units from sink.unit_ctr.
 template <typename TabT, bool FULL>
+__device__ __forceinline__ void chunk_finish_depth(const WalkParams& p, const TabT* __restrict__ tab,
+                                                   uint32_t Cs, const SurvivorSink<TabT>& sink,
+                                                   const uint4& rec, int32_t id, uint32_t s,
+                                                   int depth) {
+    if (depth == 2)
+        chunk_finish<TabT, FULL, 2>(p, tab, Cs, sink, rec, id, s);
+    else
+        chunk_finish<TabT, FULL, 1>(p, tab, Cs, sink, rec, id, s);
+}
+
+// Visits every readable bucket of state q; warps take units (readable first class,
+// block of 32 second keys) from a shared counter.  With ENUMERATE the chunks of the
+// readable buckets are written to the descriptor list (and walked later, see
+// walk_chunks); otherwise they are walked on the spot.
+template <typename TabT, bool FULL, bool ENUMERATE>
 __device__ __forceinline__ void walk_row(const WalkParams& p, const TabT* __restrict__ tab, int C,
                                          uint32_t Cs, bool two_level, const int32_t* s_gstart,
                                          const SurvivorSink<TabT>& sink, int q) {
@@ -111,7 +158,7 @@ __device__ __forceinline__ void walk_row(const WalkParams& p, const TabT* __rest
     const int U = n_live * KB;
     while (true) {
         int j = 0;
-        if (lane == 0) j = atomicAdd(sink.unit_ctr, 1);
+        if (lane == 0) j = atomicAdd(&sink.ctrs[0], 1);
         j = __shfl_sync(kFullWarp, j, 0);
         if (j >= U) break;
         const int li = j / KB, kb = j - li * KB;
@@ -142,21 +189,71 @@ __device__ __forceinline__ void walk_row(const WalkParams& p, const TabT* __rest
             cnt = s_gstart[c0 + 1] - start;
             s2 = s1;
         }
-        uint32_t m = __ballot_sync(kFullWarp, cnt > 0 && s2 != dead);
-        while (m) {
-            const int l = __ffs(m) - 1;
-            m &= m - 1;
-            const int bstart = __shfl_sync(kFullWarp, start, l);
-            const int bn = __shfl_sync(kFullWarp, cnt, l);
-            const uint32_t bs = __shfl_sync(kFullWarp, s2, l);
-            if (two_level && !(kb == 0 && l == 0)) {
-                for (int i0 = 0; i0 < bn; i0 += 32)
-                    walk_chunk<TabT, FULL, 2>(p, tab, Cs, sink, bstart + i0, bn - i0, bs, lane);
-            } else {
-                for (int i0 = 0; i0 < bn; i0 += 32)
-                    walk_chunk<TabT, FULL, 1>(p, tab, Cs, sink, bstart + i0, bn - i0, bs, lane);
+        const bool alive = cnt > 0 && s2 != dead;
+        if (ENUMERATE) {
+            const int nch = alive ? (cnt + 31) >> 5 : 0;
+            int incl = nch;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int o = __shfl_up_sync(kFullWarp, incl, off);
+                if (lane >= off) incl += o;
+            }
+            const int total = __shfl_sync(kFullWarp, incl, 31);
+            if (total == 0) continue;
+            int base = 0;
+            if (lane == 0) base = atomicAdd(&sink.ctrs[1], total);
+            base = __shfl_sync(kFullWarp, base, 0);
+            if (base + total > sink.desc_cap) {
+                if (lane == 0) sink.ctrs[3] = 1;  // the row is redone without the list
+                continue;
+            }
+            const int depth = (two_level && !(kb == 0 && lane == 0)) ? 2 : 1;
+            for (int k = 0; k < nch; ++k)
+                sink.descs[base + incl - nch + k] =
+                    Desc<TabT>::pack(start + 32 * k, s2, min(32, cnt - 32 * k), depth);
+        } else {
+            uint32_t m = __ballot_sync(kFullWarp, alive);
+            while (m) {
+                const int l = __ffs(m) - 1;
+                m &= m - 1;
+                const int bstart = __shfl_sync(kFullWarp, start, l);
+                const int bn = __shfl_sync(kFullWarp, cnt, l);
+                const uint32_t bs = __shfl_sync(kFullWarp, s2, l);
+                const int depth = (two_level && !(kb == 0 && l == 0)) ? 2 : 1;
+                for (int i0 = 0; i0 < bn; i0 += 32) {
+                    uint4 rec;
+                    int32_t id;
+                    chunk_load(p, bstart + i0, bn - i0, lane, rec, id);
+                    chunk_finish_depth<TabT, FULL>(p, tab, Cs, sink, rec, id, bs, depth);
+                }
             }
         }
+    }
+}
+
+// Walks the chunks of the descriptor list; a warp takes two at a time and issues the
+// loads of both before walking either.
+template <typename TabT, bool FULL>
+__device__ __forceinline__ void walk_chunks(const WalkParams& p, const TabT* __restrict__ tab,
+                                            uint32_t Cs, const SurvivorSink<TabT>& sink) {
+    using D = Desc<TabT>;
+    const int lane = threadIdx.x & 31;
+    const int total = sink.ctrs[1];
+    while (true) {
+        int i = 0;
+        if (lane == 0) i = atomicAdd(&sink.ctrs[2], 2);
+        i = __shfl_sync(kFullWarp, i, 0);
+        if (i >= total) break;
+        const typename D::type d0 = sink.descs[i];
+        const bool two = i + 1 < total;
+        const typename D::type d1 = sink.descs[two ? i + 1 : i];
+        uint4 rec0, rec1;
+        int32_t id0, id1;
+        chunk_load(p, D::start(d0), D::count(d0), lane, rec0, id0);
+        chunk_load(p, D::start(d1), two ? D::count(d1) : 0, lane, rec1, id1);
+        chunk_finish_depth<TabT, FULL>(p, tab, Cs, sink, rec0, id0, D::state(d0), D::depth(d0));
+        if (two)
+            chunk_finish_depth<TabT, FULL>(p, tab, Cs, sink, rec1, id1, D::state(d1), D::depth(d1));
     }
 }
 
@@ -257,7 +354,7 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
     extern __shared__ __align__(128) uint8_t smem_raw[];
     __shared__ uint64_t bar;
     __shared__ int32_t s_gstart[260];
-    __shared__ int s_unit_ctr;
+    __shared__ int s_ctrs[4];
 
     if (p.meta->any_bad != 0) {
         raw_rows<OutT, HAS_OUT>(p);
@@ -270,8 +367,10 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
     OutT* stage = reinterpret_cast<OutT*>(smem_raw + warp * kStageBytes);
     uint32_t* mwords = reinterpret_cast<uint32_t*>(smem_raw + kWalkWarps * kStageBytes) + warp * kSliceWords;
     int* counts = reinterpret_cast<int*>(smem_raw + kWalkWarps * (kStageBytes + kSliceWords * 4));
-    const size_t table_off = (kWalkWarps * (kStageBytes + kSliceWords * 4) +
-                              static_cast<size_t>(nslices) * 4 + 127) / 128 * 128;
+    const size_t desc_off = (kWalkWarps * (kStageBytes + kSliceWords * 4) +
+                             static_cast<size_t>(nslices) * 4 + 15) / 16 * 16;
+    typename Desc<TabT>::type* descs = reinterpret_cast<typename Desc<TabT>::type*>(smem_raw + desc_off);
+    const size_t table_off = (desc_off + kDescCap * sizeof(typename Desc<TabT>::type) + 127) / 128 * 128;
     TabT* stab = reinterpret_cast<TabT*>(smem_raw + table_off);
 
     const TabT* gtab = static_cast<const TabT*>(p.table);
@@ -305,7 +404,9 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
     SurvivorSink<TabT> sink;
     sink.lists = scratch + static_cast<size_t>(blockIdx.x) * nslices * kSlice;
     sink.counts = counts;
-    sink.unit_ctr = &s_unit_ctr;
+    sink.descs = descs;
+    sink.desc_cap = kDescCap;
+    sink.ctrs = s_ctrs;
 
     const int nrows = p.q_end - p.q_begin;
     for (int r = blockIdx.x; r < nrows; r += gridDim.x) {
@@ -313,12 +414,29 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
         OutT* nrow = HAS_OUT ? static_cast<OutT*>(p.next) + static_cast<size_t>(r) * p.N : nullptr;
         uint32_t* mrow = p.mask + static_cast<size_t>(r) * p.G;
         for (int i = threadIdx.x; i < nslices; i += kWalkThreads) counts[i] = 0;
-        if (threadIdx.x == 0) s_unit_ctr = 0;
+        if (threadIdx.x < 4) s_ctrs[threadIdx.x] = 0;
         __syncthreads();
         if (full)
-            walk_row<TabT, true>(p, stab, C, Cs, two_level, s_gstart, sink, q);
+            walk_row<TabT, true, true>(p, stab, C, Cs, two_level, s_gstart, sink, q);
         else
-            walk_row<TabT, false>(p, gtab, C, Cs, two_level, s_gstart, sink, q);
+            walk_row<TabT, false, true>(p, gtab, C, Cs, two_level, s_gstart, sink, q);
+        __syncthreads();  // the chunk list of the row is complete
+        if (s_ctrs[3] == 0) {
+            if (full)
+                walk_chunks<TabT, true>(p, stab, Cs, sink);
+            else
+                walk_chunks<TabT, false>(p, gtab, Cs, sink);
+        } else {
+            // more chunks than the list holds (a state that reads almost everything):
+            // walk the buckets unit by unit instead
+            __syncthreads();
+            if (threadIdx.x == 0) s_ctrs[0] = 0;
+            __syncthreads();
+            if (full)
+                walk_row<TabT, true, false>(p, stab, C, Cs, two_level, s_gstart, sink, q);
+            else
+                walk_row<TabT, false, false>(p, gtab, C, Cs, two_level, s_gstart, sink, q);
+        }
         __syncthreads();  // every survivor of the row is in its list (stores visible CTA-wide)
         assemble_row<TabT, OutT, HAS_OUT>(p, sink, stage, mwords, nslices, q, nrow, mrow);
         __syncthreads();  // counters and lists are reused by the next row
@@ -330,7 +448,8 @@ template <typename OutT, bool HAS_OUT>
 size_t sparse_fixed_smem(int32_t N) {
     const size_t nslices = (static_cast<size_t>(N) + kSlice - 1) >> kSliceShift;
     const size_t stage = HAS_OUT ? kSlice * sizeof(OutT) : 0;
-    return (kWalkWarps * (stage + kSliceWords * 4) + nslices * 4 + 127) / 128 * 128;
+    const size_t desc_off = (kWalkWarps * (stage + kSliceWords * 4) + nslices * 4 + 15) / 16 * 16;
+    return (desc_off + kDescCap * 16 + 127) / 128 * 128;  // 16 = the larger descriptor type
 }
 
 template <typename TabT, typename OutT, bool HAS_OUT>
@@ -341,9 +460,15 @@ cudaError_t launch_sparse(const WalkParams& p, void* scratch, int grid, cudaStre
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(p.smem_cap));
     if (e != cudaSuccess) return e;
+    // what is left after staging, counters and the descriptor list may hold the table
+    const size_t nslices = (static_cast<size_t>(p.N) + kSlice - 1) >> kSliceShift;
+    const size_t stage = HAS_OUT ? kSlice * sizeof(OutT) : 0;
+    const size_t desc_off = (kWalkWarps * (stage + kSliceWords * 4) + nslices * 4 + 15) / 16 * 16;
+    const size_t table_off =
+        (desc_off + kDescCap * sizeof(typename Desc<TabT>::type) + 127) / 128 * 128;
     kernel<<<grid, kWalkThreads, p.smem_cap, stream>>>(
         p, static_cast<typename Entry<TabT>::type*>(scratch),
-        static_cast<uint32_t>(p.smem_cap - fixed));
+        static_cast<uint32_t>(p.smem_cap - table_off));
     return cudaGetLastError();
 }
 
