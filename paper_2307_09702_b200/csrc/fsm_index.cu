@@ -7,7 +7,7 @@
 //   3. prepare_inputs  class-compressed table [Q x Cs] with exact verification that every
 //                      byte's column equals its class representative's column; token
 //                      records (dense walk) or bucket counts (sparse walk)
-//   3b. sort_tokens    sparse walk only: tokens sorted by (first, second) byte class
+//   3b. scan_keys, sort_tokens   sparse walk only: tokens sorted by (first, second) byte class
 //   4. walk            dense: every (state, token) pair walked by warp tiles;
 //      walk_sparse     only tokens of readable buckets walked, rows pre-filled with dead
 // If verification in 3 fails (a 64-bit hash collision) the walk reads the uncompressed
@@ -67,10 +67,10 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
                         sparse_fixed_smem<int32_t, true>(N) + 4096 <= static_cast<size_t>(dev.smem_optin - 2048);
 
     const int hash_blocks = Q < kHashBlocks ? Q : kHashBlocks;
-    hash_columns<<<hash_blocks, 256, 0, stream>>>(dfa_trans, Q, dead_state, ws.partial,
-                                                  tune.weak_hash, status_word);
-    derive_classes<<<1, 256, 0, stream>>>(ws.partial, hash_blocks, ws.meta, ws.cls, ws.class_rep,
-                                          ws.gcount, ws.count2, ws.cursor2);
+    hash_columns<<<hash_blocks, 256 * kHashRowLanes, 0, stream>>>(
+        dfa_trans, Q, dead_state, ws.partial, tune.weak_hash, ws.gcount, ws.count2, ws.cursor2,
+        status_word);
+    derive_classes<<<1, 256, 0, stream>>>(ws.partial, hash_blocks, ws.meta, ws.cls, ws.class_rep);
     const int row_blocks = Q < 2 * dev.sm_count ? Q : 2 * dev.sm_count;
     const int tok_blocks = (G * 32 + 255) / 256;
     int32_t* count_into = sparse ? ws.count2 : nullptr;
@@ -85,10 +85,11 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
             row_blocks, ws.meta, ws.cls, ws.class_rep, static_cast<uint16_t*>(ws.table),
             ws.tok_cls, ws.tok_len, ws.gcount, count_into, status_word);
     if (sparse) {
-        const int place_blocks = (N + 255) / 256;
-        sort_tokens<<<place_blocks + kTwoLevelMaxC + 1, 256, 0, stream>>>(
-            vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, place_blocks, ws.meta, ws.cls,
-            ws.gcount, ws.count2, ws.cursor2, ws.gstart, ws.start2, ws.srec, ws.sid);
+        scan_keys<<<kTwoLevelMaxC + 1, 256, 0, stream>>>(ws.meta, ws.gcount, ws.count2, ws.gstart,
+                                                         ws.start2);
+        sort_tokens<<<(N + 255) / 256, 256, 0, stream>>>(vocab_bytes, vocab_offsets, vocab_nbytes,
+                                                         N, eos_id, ws.meta, ws.cls, ws.start2,
+                                                         ws.cursor2, ws.srec, ws.sid);
     }
     if (cudaGetLastError() != cudaSuccess) return FSM_ERR_CUDA;
 

@@ -7,45 +7,55 @@ namespace fsm {
 namespace {
 
 // ---------------------------------------------------------------------------- 1
-// Thread b owns byte column b of delta; a block strides over rows (coalesced 1 KB row
-// reads).  The per-column hash is a wrap-around sum of mixed (row, value) pairs, so
-// equal columns hash alike and partial sums from different blocks simply add.
-__global__ void __launch_bounds__(256) hash_columns(const int32_t* __restrict__ trans, int32_t Q,
-                                                   int32_t dead, uint64_t* __restrict__ partial,
-                                                   int weak, int32_t* status) {
-    const int b = threadIdx.x;
+// Thread (b, lane) owns byte column b of delta for rows lane, lane+4, ... of the block's
+// share (coalesced 1 KB row reads).  The per-column hash is a wrap-around sum of mixed
+// (row, value) pairs, so equal columns hash alike and partial sums simply add.  The
+// blocks also clear the counters of the token sort.
+constexpr int kHashRowLanes = 4;
+
+__global__ void __launch_bounds__(256 * kHashRowLanes)
+hash_columns(const int32_t* __restrict__ trans, int32_t Q, int32_t dead,
+             uint64_t* __restrict__ partial, int weak, int32_t* __restrict__ gcount,
+             int32_t* __restrict__ count2, int32_t* __restrict__ cursor2, int32_t* status) {
+    __shared__ uint64_t part[kHashRowLanes][256];
+    const int b = threadIdx.x & 255, rl = threadIdx.x >> 8;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < kKeys; i += gridDim.x * blockDim.x) {
+        count2[i] = 0;
+        cursor2[i] = 0;
+        if (i < 256) gcount[i] = 0;
+    }
     uint64_t h = 0;
     bool bad = false;
-    for (int q = blockIdx.x; q < Q; q += gridDim.x) {
+    for (int q = blockIdx.x * kHashRowLanes + rl; q < Q; q += gridDim.x * kHashRowLanes) {
         if (q == dead) continue;
         int32_t v = trans[static_cast<size_t>(q) * 256 + b];
         bad |= static_cast<uint32_t>(v) >= static_cast<uint32_t>(Q);
         h += mix64((static_cast<uint64_t>(q) << 32) | static_cast<uint32_t>(v));
     }
-    partial[blockIdx.x * 256 + b] = weak ? 0 : h;
-    if (__syncthreads_or(bad) && threadIdx.x == 0) raise_flag(status, FSM_FLAG_TRANS_RANGE);
+    part[rl][b] = h;
+    const int any_bad = __syncthreads_or(bad);
+    if (rl == 0) {
+        uint64_t sum = 0;
+#pragma unroll
+        for (int k = 0; k < kHashRowLanes; ++k) sum += part[k][b];
+        partial[blockIdx.x * 256 + b] = weak ? 0 : sum;
+    }
+    if (any_bad && threadIdx.x == 0) raise_flag(status, FSM_FLAG_TRANS_RANGE);
 }
 
 // ---------------------------------------------------------------------------- 2
 // One block.  Bytes whose column hashes are equal form a class, represented by the
 // smallest such byte; class ids are the ranks of the representatives.  Equal hashes
-// are found through a small open-addressing table in shared memory.  Also clears the
-// counters of the token sort.
+// are found through a small open-addressing table in shared memory.
 __global__ void __launch_bounds__(256) derive_classes(const uint64_t* __restrict__ partial,
                                                      int nblocks, IndexMeta* meta, uint8_t* cls,
-                                                     uint8_t* class_rep, int32_t* gcount,
-                                                     int32_t* count2, int32_t* cursor2) {
+                                                     uint8_t* class_rep) {
     constexpr int kSlots = 1024;
     __shared__ unsigned long long keys[kSlots];
     __shared__ int min_byte[kSlots];
     __shared__ uint32_t rep_bits[8];
     constexpr unsigned long long kEmpty = ~0ull;
     const int b = threadIdx.x;
-    gcount[b] = 0;
-    for (int i = b; i < kKeys; i += 256) {
-        count2[i] = 0;
-        cursor2[i] = 0;
-    }
     uint64_t sum = 0;
 #pragma unroll 8
     for (int k = 0; k < nblocks; ++k) sum += partial[k * 256 + b];
@@ -132,9 +142,12 @@ prepare_inputs(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vo
         const bool two = meta->two_level != 0;
         const int64_t v = static_cast<int64_t>(blockIdx.x - row_blocks) * 256 + threadIdx.x;
         const TokenInfo t = token_info(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, s_cls, v, &bad);
+        // one atomic per distinct key of the warp
+        const int key = t.len > 0 ? bucket_key(two, t.first, t.second_key) : -1;
+        const uint32_t peers = __match_any_sync(kFullWarp, key);
         if (t.len > 0) {
             atomicAdd(&hist[t.first], 1);
-            atomicAdd(&count2[bucket_key(two, t.first, t.second_key)], 1);
+            if ((threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&count2[key], __popc(peers));
         }
         if (__syncthreads_or(bad) && threadIdx.x == 0) raise_flag(status, FSM_FLAG_OFFSETS);
         if (hist[threadIdx.x] > 0) atomicAdd(&gcount[threadIdx.x], hist[threadIdx.x]);
@@ -164,19 +177,16 @@ prepare_inputs(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vo
 // ---------------------------------------------------------------------------- 3b
 // Token order of the sparse walk: a counting sort by bucket key - the class of the
 // first byte and, when there are at most kTwoLevelMaxC classes, the class of the second
-// byte (key 0 = one-byte token).  Blocks [0, token_blocks) place 256 tokens each; the
-// remaining blocks publish the first sorted position of every key (start2).  A record
-// keeps the length and the classes of bytes 1..15; `sid` holds the token id.
+// byte (key 0 = one-byte token).  scan_keys turns the counts into first positions
+// (block c0 handles the keys of first class c0); sort_tokens places 256 tokens per
+// block.  A record keeps the length and the classes of bytes 1..15; `sid` holds the
+// token id.
 __global__ void __launch_bounds__(256)
-sort_tokens(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vocab_offsets,
-            int64_t vocab_nbytes, int32_t N, int32_t eos_id, int token_blocks,
-            const IndexMeta* __restrict__ meta, const uint8_t* __restrict__ cls,
-            const int32_t* __restrict__ gcount, const int32_t* __restrict__ count2,
-            int32_t* __restrict__ cursor2, int32_t* __restrict__ gstart,
-            int32_t* __restrict__ start2, uint4* __restrict__ srec, int32_t* __restrict__ sid) {
+scan_keys(const IndexMeta* __restrict__ meta, const int32_t* __restrict__ gcount,
+          const int32_t* __restrict__ count2, int32_t* __restrict__ gstart,
+          int32_t* __restrict__ start2) {
     __shared__ int gst[257];
-    __shared__ uint8_t s_cls[256];
-    s_cls[threadIdx.x] = cls[threadIdx.x];
+    __shared__ int wsum[8];
     if (threadIdx.x < 32) {  // exclusive prefix over the 256 class counts, 8 per lane
         int local[8], sum = 0;
 #pragma unroll
@@ -195,35 +205,55 @@ sort_tokens(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__
         if (threadIdx.x == 31) gst[256] = incl;
     }
     __syncthreads();
-    const bool two = meta->two_level != 0;
+    const int c0 = blockIdx.x;
+    if (c0 == 0) {
+        gstart[threadIdx.x] = gst[threadIdx.x];
+        if (threadIdx.x == 0) gstart[256] = gst[256];
+    }
     const int C = meta->C;
-    if (static_cast<int>(blockIdx.x) >= token_blocks) {
-        const int c0 = blockIdx.x - token_blocks;
-        if (c0 == 0) {
-            gstart[threadIdx.x] = gst[threadIdx.x];
-            if (threadIdx.x == 0) gstart[256] = gst[256];
-        }
-        if (two) {
-            if (c0 < C && static_cast<int>(threadIdx.x) <= C) {
-                int before = 0;
-                for (int k = 0; k < static_cast<int>(threadIdx.x); ++k)
-                    before += count2[c0 * kKeyStride + k];
-                start2[c0 * kKeyStride + threadIdx.x] = gst[c0] + before;
-            }
-        } else if (c0 == 0) {
-            start2[threadIdx.x] = gst[threadIdx.x];
-        }
+    if (meta->two_level == 0) {
+        if (c0 == 0) start2[threadIdx.x] = gst[threadIdx.x];
         return;
     }
+    if (c0 >= C) return;
+    // exclusive prefix over the C + 1 <= 128 keys of first class c0
+    const int t = threadIdx.x;
+    const int mine = t <= C ? count2[c0 * kKeyStride + t] : 0;
+    int incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int o = __shfl_up_sync(kFullWarp, incl, off);
+        if ((t & 31) >= off) incl += o;
+    }
+    if ((t & 31) == 31) wsum[t >> 5] = incl;
+    __syncthreads();
+    int before = 0;
+    for (int w = 0; w < (t >> 5); ++w) before += wsum[w];
+    if (t <= C) start2[c0 * kKeyStride + t] = gst[c0] + before + incl - mine;
+}
+
+__global__ void __launch_bounds__(256)
+sort_tokens(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vocab_offsets,
+            int64_t vocab_nbytes, int32_t N, int32_t eos_id, const IndexMeta* __restrict__ meta,
+            const uint8_t* __restrict__ cls, const int32_t* __restrict__ start2,
+            int32_t* __restrict__ cursor2, uint4* __restrict__ srec, int32_t* __restrict__ sid) {
+    __shared__ uint8_t s_cls[256];
+    s_cls[threadIdx.x] = cls[threadIdx.x];
+    __syncthreads();
+    const bool two = meta->two_level != 0;
     bool bad = false;
     const int64_t v = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
     const TokenInfo t = token_info(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, s_cls, v, &bad);
+    // one cursor atomic per distinct key of the warp
+    const int key = t.len > 0 ? bucket_key(two, t.first, t.second_key) : -1;
+    const uint32_t peers = __match_any_sync(kFullWarp, key);
+    const int lane = threadIdx.x & 31;
+    const int leader = __ffs(peers) - 1;
+    int base = 0;
+    if (t.len > 0 && lane == leader) base = atomicAdd(&cursor2[key], __popc(peers));
+    base = __shfl_sync(kFullWarp, base, leader);
     if (t.len > 0) {
-        int before = 0;
-        if (two)
-            for (int k = 0; k < t.second_key; ++k) before += count2[t.first * kKeyStride + k];
-        const int pos = gst[t.first] + before +
-                        atomicAdd(&cursor2[bucket_key(two, t.first, t.second_key)], 1);
+        const int pos = start2[key] + base + __popc(peers & ((1u << lane) - 1u));
         uint32_t w[4] = {static_cast<uint32_t>(t.len), 0, 0, 0};
         const int nb = min(t.len, kInlineBytes);
         for (int i = 1; i < nb; ++i)

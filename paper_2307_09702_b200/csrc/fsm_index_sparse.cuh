@@ -269,49 +269,64 @@ __device__ __forceinline__ void assemble_row(const WalkParams& p, const Survivor
     const uint4 dead16 = make_uint4(d32, d32, d32, d32);
     constexpr int kVec = 16 / sizeof(OutT);          // elements per 16-byte vector
     constexpr int kVecPerLane = kSlice / kVec / 32;  // 2 (int32) or 1 (uint16)
-    const bool eos_ok = p.eos_id >= 0 && q != p.dead && p.accept[q];
+    // a slice is a whole number of 16-byte vectors, so every slice of an aligned row is aligned
+    const bool vec_ok = HAS_OUT && (reinterpret_cast<uintptr_t>(nrow) & 15) == 0;
+    const int eos_slice =
+        (p.eos_id >= 0 && q != p.dead && p.accept[q]) ? (p.eos_id >> kSliceShift) : -1;
+    const int last_full = p.N >> kSliceShift;  // slices below this index are complete
+    const typename E::type* lst = sink.lists + static_cast<size_t>(warp) * kSlice;
+    OutT* dst = HAS_OUT ? nrow + warp * kSlice : nullptr;
+    uint32_t* mdst = mrow + warp * kSliceWords;
+    uint4* stage4 = reinterpret_cast<uint4*>(stage);
     for (int sl = warp; sl < nslices; sl += kWalkWarps) {
-        const int base = sl << kSliceShift;
-        const int n = min(kSlice, p.N - base);
         const int cnt = sink.counts[sl];
         // the first 32 survivors are fetched before the fill to overlap their latency
         typename E::type e0 = 0;
-        if (lane < cnt) e0 = sink.lists[static_cast<size_t>(sl) * kSlice + lane];
+        if (lane < cnt) e0 = lst[lane];
         if (HAS_OUT) {
 #pragma unroll
-            for (int k = 0; k < kVecPerLane; ++k)
-                reinterpret_cast<uint4*>(stage)[lane + 32 * k] = dead16;
+            for (int k = 0; k < kVecPerLane; ++k) stage4[lane + 32 * k] = dead16;
         }
         if (lane < kSliceWords) mwords[lane] = 0;
         __syncwarp();
         if (lane < cnt) {
-            if (HAS_OUT) stage[E::lid(e0)] = static_cast<OutT>(E::state(e0));
-            atomicOr(&mwords[E::lid(e0) >> 5], 1u << (E::lid(e0) & 31));
+            const uint32_t lid = E::lid(e0);
+            if (HAS_OUT) stage[lid] = static_cast<OutT>(E::state(e0));
+            atomicOr(&mwords[lid >> 5], 1u << (lid & 31));
         }
         for (int i = 32 + lane; i < cnt; i += 32) {
-            const typename E::type e = sink.lists[static_cast<size_t>(sl) * kSlice + i];
-            if (HAS_OUT) stage[E::lid(e)] = static_cast<OutT>(E::state(e));
-            atomicOr(&mwords[E::lid(e) >> 5], 1u << (E::lid(e) & 31));
+            const typename E::type e = lst[i];
+            const uint32_t lid = E::lid(e);
+            if (HAS_OUT) stage[lid] = static_cast<OutT>(E::state(e));
+            atomicOr(&mwords[lid >> 5], 1u << (lid & 31));
         }
-        if (eos_ok && lane == 0 && p.eos_id >= base && p.eos_id < base + n) {
-            const int e = p.eos_id - base;
+        if (sl == eos_slice && lane == 0) {
+            const int e = p.eos_id & (kSlice - 1);
             if (HAS_OUT) stage[e] = static_cast<OutT>(q);
             atomicOr(&mwords[e >> 5], 1u << (e & 31));
         }
         __syncwarp();
-        if (lane < (n + 31) / 32) mrow[(base >> 5) + lane] = mwords[lane];
-        if (HAS_OUT) {
-            OutT* dst = nrow + base;
-            if (n == kSlice && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+        if (sl < last_full) {
+            if (lane < kSliceWords) mdst[lane] = mwords[lane];
+            if (HAS_OUT) {
+                if (vec_ok) {
 #pragma unroll
-                for (int k = 0; k < kVecPerLane; ++k)
-                    reinterpret_cast<uint4*>(dst)[lane + 32 * k] =
-                        reinterpret_cast<const uint4*>(stage)[lane + 32 * k];
-            } else {  // ragged last slice or unaligned row: element-wise, still coalesced
-                for (int i = lane; i < n; i += 32) dst[i] = stage[i];
+                    for (int k = 0; k < kVecPerLane; ++k)
+                        reinterpret_cast<uint4*>(dst)[lane + 32 * k] = stage4[lane + 32 * k];
+                } else {  // unaligned row: element-wise, still coalesced
+                    for (int i = lane; i < kSlice; i += 32) dst[i] = stage[i];
+                }
             }
+        } else {  // ragged last slice
+            const int n = p.N - (sl << kSliceShift);
+            if (lane < (n + 31) / 32) mdst[lane] = mwords[lane];
+            if (HAS_OUT)
+                for (int i = lane; i < n; i += 32) dst[i] = stage[i];
         }
         __syncwarp();  // staging is refilled by the next slice
+        lst += static_cast<size_t>(kWalkWarps) * kSlice;
+        if (HAS_OUT) dst += kWalkWarps * kSlice;
+        mdst += kWalkWarps * kSliceWords;
     }
 }
 
