@@ -278,11 +278,16 @@ __device__ __forceinline__ void assemble_row(const WalkParams& p, const Survivor
     OutT* dst = HAS_OUT ? nrow + warp * kSlice : nullptr;
     uint32_t* mdst = mrow + warp * kSliceWords;
     uint4* stage4 = reinterpret_cast<uint4*>(stage);
+    // The first 32 survivors of a slice are fetched one slice ahead, so that the trip to
+    // the L2-resident scratch overlaps the assembly of the previous slice.
+    int cnt = warp < nslices ? sink.counts[warp] : 0;
+    typename E::type e0 = 0;
+    if (lane < cnt) e0 = lst[lane];
     for (int sl = warp; sl < nslices; sl += kWalkWarps) {
-        const int cnt = sink.counts[sl];
-        // the first 32 survivors are fetched before the fill to overlap their latency
-        typename E::type e0 = 0;
-        if (lane < cnt) e0 = lst[lane];
+        const int next = sl + kWalkWarps;
+        const int cnt_next = next < nslices ? sink.counts[next] : 0;
+        typename E::type e_next = 0;
+        if (lane < cnt_next) e_next = lst[static_cast<size_t>(kWalkWarps) * kSlice + lane];
         if (HAS_OUT) {
 #pragma unroll
             for (int k = 0; k < kVecPerLane; ++k) stage4[lane + 32 * k] = dead16;
@@ -324,6 +329,8 @@ __device__ __forceinline__ void assemble_row(const WalkParams& p, const Survivor
                 for (int i = lane; i < n; i += 32) dst[i] = stage[i];
         }
         __syncwarp();  // staging is refilled by the next slice
+        cnt = cnt_next;
+        e0 = e_next;
         lst += static_cast<size_t>(kWalkWarps) * kSlice;
         if (HAS_OUT) dst += kWalkWarps * kSlice;
         mdst += kWalkWarps * kSliceWords;
