@@ -53,37 +53,67 @@ template <> struct Elem<uint32_t> {  // fp32 bit patterns
     static constexpr int kPerWord = 1;
     static constexpr uint32_t kNegInfWord = 0xFF800000u;
     __device__ static float get(uint32_t w, int) { return __uint_as_float(w); }
+    // keeps the allowed element, -inf otherwise
     __device__ static uint32_t select(uint32_t w, uint32_t bits) { return (bits & 1u) ? w : kNegInfWord; }
+    // largest value of a masked vector of NW words
+    template <int NW>
+    __device__ static float vmax(const uint32_t (&w)[NW]) {
+        float m = __uint_as_float(w[0]);
+#pragma unroll
+        for (int i = 1; i < NW; ++i) m = fmaxf(m, __uint_as_float(w[i]));
+        return m;
+    }
 };
-template <> struct Elem<uint16_t> {  // bf16 bit patterns
+template <> struct Elem<uint16_t> {  // bf16 bit patterns, two per word
     static constexpr int kPerWord = 2;
     static constexpr uint32_t kNegInfWord = 0xFF80FF80u;
     __device__ static float get(uint32_t w, int j) { return __uint_as_float(j ? (w & 0xFFFF0000u) : (w << 16)); }
+    // one byte permute per word: allowed halves come from w, the others from -inf
     __device__ static uint32_t select(uint32_t w, uint32_t bits) {
-        const uint32_t keep = ((bits & 1u) ? 0x0000FFFFu : 0u) | ((bits & 2u) ? 0xFFFF0000u : 0u);
-        return (w & keep) | (kNegInfWord & ~keep);
+        const uint32_t sel = 0x7654u ^ ((bits & 1u) * 0x0044u) ^ ((bits & 2u) * 0x2200u);
+        return __byte_perm(w, kNegInfWord, sel);
+    }
+    template <int NW>
+    __device__ static float vmax(const uint32_t (&w)[NW]) {
+        uint32_t m = w[0];
+#pragma unroll
+        for (int i = 1; i < NW; ++i) asm("max.bf16x2 %0, %0, %1;" : "+r"(m) : "r"(w[i]));
+        return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
     }
 };
 
-// Processes one vector of NW 32-bit words whose first element has index e0.
+// Running maximum of one thread.  The position inside the winning vector is not
+// tracked while streaming: the vector's index and bitmask bits are kept and the
+// position is found once, at the end (see locate()).
+struct ThreadBest {
+    float val;      // NaN until the first vector with an allowed entry
+    int vec;        // index of the vector that holds it, -1 = none
+    uint32_t bits;  // allowed bits of that vector
+};
+
+// Masks one vector of NW words in place and folds its maximum into `tb`.
 template <typename T, int NW>
-__device__ __forceinline__ void process(uint32_t (&w)[NW], uint32_t bits, int e0, Best& best) {
+__device__ __forceinline__ void process(uint32_t (&w)[NW], uint32_t bits, int vec, ThreadBest& tb) {
     constexpr int PW = Elem<T>::kPerWord;
 #pragma unroll
-    for (int i = 0; i < NW; ++i) {
-        const uint32_t b = (bits >> (i * PW)) & ((1u << PW) - 1u);
-#pragma unroll
-        for (int j = 0; j < PW; ++j) {
-            if (b & (1u << j)) {
-                const float x = Elem<T>::get(w[i], j);
-                if (!(x <= best.val)) {  // also true for the first allowed entry (val is NaN)
-                    best.val = x;
-                    best.idx = e0 + i * PW + j;
-                }
-            }
-        }
-        w[i] = Elem<T>::select(w[i], b);
+    for (int i = 0; i < NW; ++i) w[i] = Elem<T>::select(w[i], (bits >> (i * PW)) & ((1u << PW) - 1u));
+    const float m = Elem<T>::template vmax<NW>(w);
+    if (!(m <= tb.val)) {  // strictly larger, or the first allowed entries (val is NaN)
+        tb.val = m;
+        tb.vec = vec;
+        tb.bits = bits;
     }
+}
+
+// Lowest allowed position of a vector whose value equals `val` (IEEE equality).
+template <typename T, int NW>
+__device__ __forceinline__ int locate(const uint32_t (&w)[NW], uint32_t bits, float val) {
+    constexpr int PW = Elem<T>::kPerWord;
+    int pos = NW * PW;
+#pragma unroll
+    for (int j = NW * PW - 1; j >= 0; --j)
+        if (((bits >> j) & 1u) && Elem<T>::get(w[j / PW], j % PW) == val) pos = j;
+    return pos;
 }
 
 template <typename T, bool WRITE>
@@ -111,25 +141,48 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
     T* out = WRITE ? static_cast<T*>(p.out) + static_cast<size_t>(row) * p.row_stride : nullptr;
     const bool wide = ((reinterpret_cast<uintptr_t>(in) | (WRITE ? reinterpret_cast<uintptr_t>(out) : 0)) & 31) == 0;
 
-    Best best{__int_as_float(0x7FC00000), kNone};
+    ThreadBest tb{__int_as_float(0x7FC00000), -1, 0u};
     const int tid = rank * kStepThreads + threadIdx.x;
     const int nthreads = k * kStepThreads;
 
     int done = 0;  // elements covered by whole vectors
     if (wide) {
+        // Per thread and pass: the bitmask bits of kGroup vectors are fetched first (one
+        // round trip to L2), then the vectors are streamed kUnroll at a time - every needed
+        // logits load of a batch is issued before any arithmetic, so that several 32-byte
+        // loads are in flight per thread.
+        constexpr int kUnroll = 4, kGroup = 8;
         const int nvec = p.N / EPV;
-        for (int vi = tid; vi < nvec; vi += nthreads) {
-            const int e0 = vi * EPV;
-            const uint32_t bits = live & (mrow[e0 >> 5] >> (e0 & 31)) & ((EPV == 32) ? 0xFFFFFFFFu : ((1u << EPV) - 1u));
-            Vec32B v;
-            if (bits != 0) {
-                v = ldg_stream_32B(in + e0);
-                process<T, 8>(v.w, bits, e0, best);
-            } else {
+        constexpr uint32_t kBitsMask = (EPV == 32) ? 0xFFFFFFFFu : ((1u << EPV) - 1u);
+        for (int g0 = tid; g0 < nvec; g0 += nthreads * kGroup) {
+            uint32_t bits[kGroup];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) v.w[i] = Elem<T>::kNegInfWord;
+            for (int u = 0; u < kGroup; ++u) {
+                const int vi = g0 + u * nthreads;
+                const int e0 = vi * EPV;
+                bits[u] = vi < nvec ? (live & (__ldg(mrow + (e0 >> 5)) >> (e0 & 31)) & kBitsMask) : 0u;
             }
-            if (WRITE) stg_32B(out + e0, v);
+#pragma unroll
+            for (int h = 0; h < kGroup; h += kUnroll) {
+                Vec32B v[kUnroll];
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u)
+                    if (bits[h + u] != 0)
+                        v[u] = ldg_stream_32B(in + static_cast<size_t>(g0 + (h + u) * nthreads) * EPV);
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) {
+                    const int vi = g0 + (h + u) * nthreads;
+                    if (vi < nvec) {
+                        if (bits[h + u] != 0) {
+                            process<T, 8>(v[u].w, bits[h + u], vi, tb);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) v[u].w[i] = Elem<T>::kNegInfWord;
+                        }
+                        if (WRITE) stg_32B(out + static_cast<size_t>(vi) * EPV, v[u]);
+                    }
+                }
+            }
         }
         done = nvec * EPV;
     } else {
@@ -141,7 +194,7 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
             if (bits != 0) {
                 const uint4 v = *reinterpret_cast<const uint4*>(in + e0);
                 w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
-                process<T, 4>(w, bits, e0, best);
+                process<T, 4>(w, bits, vi, tb);
             } else {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) w[i] = Elem<T>::kNegInfWord;
@@ -149,6 +202,22 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
             if (WRITE) *reinterpret_cast<uint4*>(out + e0) = make_uint4(w[0], w[1], w[2], w[3]);
         }
         done = nvec * EPH;
+    }
+    // Position of the thread's maximum: re-read the winning vector (the allowed entries
+    // are unchanged by the masking, wherever it was written) and take the lowest
+    // allowed position that holds the value.
+    Best best{0.0f, kNone};
+    if (tb.vec >= 0) {
+        const T* src = (WRITE ? static_cast<const T*>(out) : in);
+        best.val = tb.val;
+        if (wide) {
+            Vec32B v = ldg_stream_32B(src + static_cast<size_t>(tb.vec) * EPV);
+            best.idx = tb.vec * EPV + locate<T, 8>(v.w, tb.bits, tb.val);
+        } else {
+            const uint4 v = *reinterpret_cast<const uint4*>(src + static_cast<size_t>(tb.vec) * EPH);
+            uint32_t w[4] = {v.x, v.y, v.z, v.w};
+            best.idx = tb.vec * EPH + locate<T, 4>(w, tb.bits, tb.val);
+        }
     }
     // Ragged tail (fewer elements than one vector): one element per thread of the last CTA.
     if (rank == k - 1) {
@@ -159,7 +228,7 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
             if (allowed) {
                 const float x = sizeof(T) == 4 ? __uint_as_float(static_cast<uint32_t>(raw))
                                                : __uint_as_float(static_cast<uint32_t>(raw) << 16);
-                if (!(x <= best.val)) {
+                if (best.idx == kNone || x > best.val) {  // tail ids exceed every vector id
                     best.val = x;
                     best.idx = e;
                 }
@@ -172,7 +241,6 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
 
     // A thread's own ids only grow, so its (val, idx) already holds the lowest id
     // among equal values; combining needs the full ordering.
-    if (best.idx == kNone) best.val = 0.0f;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
         Best o;

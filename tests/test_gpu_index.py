@@ -110,6 +110,29 @@ def test_two_state_automaton_and_extremes():
     check_index(trans, np.array([0, 1], dtype=np.uint8), vb, vo, 0, eos=3)
 
 
+def test_state_that_reads_everything_over_a_large_vocabulary():
+    """A state whose every byte loops: all 128,000 non-empty tokens survive, which is
+    more 32-token chunks than the sparse walk keeps descriptors for (it then walks the
+    buckets unit by unit) and fills every survivor list to the brim."""
+    w = make_config(3)
+    trans = np.full((3, 256), 2, dtype=np.int32)
+    trans[0, :] = 0                       # state 0 reads everything and stays
+    trans[1, 97:123] = 0                  # state 1 reads lowercase letters only
+    accept = np.array([1, 0, 0], dtype=np.uint8)
+    mask, nxt = check_index(trans, accept, w.vocab_bytes, w.vocab_offsets, 2, w.eos_id)
+    lens = np.diff(w.vocab_offsets)
+    assert int(np.unpackbits(mask[0].view(np.uint8)).sum()) == int((lens > 0).sum()) + 1
+
+
+def test_more_than_127_byte_classes_uses_one_level_buckets():
+    d, cls = random_class_dfa(33, n_live=300, n_classes=220, live_classes_per_state=60)
+    assert len(np.unique(d.trans.T, axis=0)) > 127
+    rng = np.random.default_rng(2)
+    toks = [bytes(rng.integers(0, 256, size=rng.integers(0, 6)).tolist()) for _ in range(5000)]
+    vb, vo = vocab_from_strings(toks)
+    check_index(d.trans, d.accept, vb, vo, d.dead, eos=77)
+
+
 def test_dead_row_contents_ignored():
     w = make_config(1)
     t = w.dfa.trans.copy()
