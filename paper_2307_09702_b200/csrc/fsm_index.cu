@@ -63,8 +63,8 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     if (tune.smem_table_cap > 0 && tune.smem_table_cap < cap) cap = tune.smem_table_cap;
     // The sparse walk needs the survivor scratch and room for its per-warp staging.
     const bool sparse = tune.walk_algo != 1 && !dense_only &&
-                        (N + kSlice - 1) / kSlice <= kMaxSlices &&
-                        sparse_fixed_smem<int32_t, true>(N) + 4096 <= static_cast<size_t>(dev.smem_optin - 2048);
+                        (N + 255) / 256 <= kMaxSlices &&
+                        sparse_table_offset<int32_t>(N) + 4096 <= static_cast<size_t>(dev.smem_optin - 2048);
 
     const int hash_blocks = Q < kHashBlocks ? Q : kHashBlocks;
     hash_columns<<<hash_blocks, 256 * kHashRowLanes, 0, stream>>>(
@@ -118,7 +118,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     p.mask = allowed_mask;
     p.next = next_state;
     p.status = status_word;
-    const int min_cap = sparse ? static_cast<int>(sparse_fixed_smem<int32_t, true>(N)) + 4096
+    const int min_cap = sparse ? static_cast<int>(sparse_table_offset<int32_t>(N)) + 4096
                                : kChunk * kMaxCs * 4;
     if (cap < min_cap) cap = min_cap;
     p.smem_cap = static_cast<uint32_t>(cap) / 128 * 128;

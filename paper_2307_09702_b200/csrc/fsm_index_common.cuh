@@ -79,7 +79,7 @@ inline Workspace carve(void* base, int32_t Q, int32_t N) {
     w.start2 = reinterpret_cast<int32_t*>(take(kKeys * sizeof(int32_t)));
     w.dense_bytes = off;
     const size_t ctas = Q < kMaxSparseCtas ? Q : kMaxSparseCtas;
-    const size_t slice_slots = (static_cast<size_t>(N) + 255) / 256 * 256;
+    const size_t slice_slots = (static_cast<size_t>(N) + 511) / 512 * 512;
     w.survivors = take(ctas * slice_slots * (Q <= 65535 ? 4 : 8));
     w.bytes = off;
     return w;

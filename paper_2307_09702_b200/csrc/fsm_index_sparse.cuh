@@ -28,9 +28,14 @@
 namespace fsm {
 namespace {
 
-constexpr int kSliceShift = 8;
-constexpr int kSlice = 1 << kSliceShift;  // token ids per assembly slice
-constexpr int kSliceWords = kSlice / 32;
+// An assembly slice is 1 KB of table-width states: 512 token ids with 16-bit table
+// entries, 256 with 32-bit entries.
+constexpr int kStageBytes = 1024;
+template <typename TabT> struct Slice {
+    static constexpr int kShift = sizeof(TabT) == 2 ? 9 : 8;
+    static constexpr int kTokens = 1 << kShift;
+};
+constexpr int kMaxSliceTokens = 512;
 constexpr int kMaxSlices = 8192;          // vocabularies up to 2 M tokens (else the dense walk)
 constexpr int kDescCap = 4096;            // chunk descriptors kept per row
 
@@ -76,7 +81,7 @@ template <> struct Desc<int32_t> {
 // Shared state of the row being walked.
 template <typename TabT>
 struct SurvivorSink {
-    typename Entry<TabT>::type* lists;  // [nslices][kSlice], this CTA's part of the scratch
+    typename Entry<TabT>::type* lists;  // [nslices][slice tokens], this CTA's part of the scratch
     int* counts;                        // [nslices], shared memory
     typename Desc<TabT>::type* descs;   // [desc_cap] chunk descriptors, shared memory
     int desc_cap;
@@ -108,10 +113,10 @@ __device__ __forceinline__ void chunk_finish(const WalkParams& p, const TabT* __
     if (go)  // longer than the inline record and still alive: finish on the raw bytes
         st = raw_walk(p, st, p.vocab_offsets[id], p.vocab_offsets[id + 1], kInlineBytes);
     if (id >= 0 && st != dead) {
-        const int slice = id >> kSliceShift;
-        const int at = atomicAdd(&sink.counts[slice], 1);  // < kSlice: a token survives once
-        sink.lists[static_cast<size_t>(slice) * kSlice + at] =
-            Entry<TabT>::pack(id & (kSlice - 1), st);
+        constexpr int kTok = Slice<TabT>::kTokens;
+        const int slice = id >> Slice<TabT>::kShift;
+        const int at = atomicAdd(&sink.counts[slice], 1);  // < kTok: a token survives once
+        sink.lists[static_cast<size_t>(slice) * kTok + at] = Entry<TabT>::pack(id & (kTok - 1), st);
     }
 }
 
@@ -258,25 +263,32 @@ __device__ __forceinline__ void walk_chunks(const WalkParams& p, const TabT* __r
 }
 
 // Assembles and stores the slices of one row; warp w takes slices w, w+32, ...
+// The slice is staged in table-entry width (1 KB per warp): filled with `dead`, then
+// the survivors are written into it.  Each lane then reads back two 16-byte vectors,
+// derives their bitmask bits from "state != dead" (a warp reduce joins the lanes of a
+// word), widens the states if the output is wider than the table entries, and stores.
 template <typename TabT, typename OutT, bool HAS_OUT>
 __device__ __forceinline__ void assemble_row(const WalkParams& p, const SurvivorSink<TabT>& sink,
-                                             OutT* stage, uint32_t* mwords, int nslices, int q,
-                                             OutT* nrow, uint32_t* mrow) {
+                                             TabT* stage, int nslices, int q, OutT* nrow,
+                                             uint32_t* mrow) {
     using E = Entry<TabT>;
+    constexpr int kTok = Slice<TabT>::kTokens;
+    constexpr int kShift = Slice<TabT>::kShift;
+    constexpr int kPerVec = 16 / sizeof(TabT);     // states per 16-byte staging vector
+    constexpr int kLanesPerWord = 32 / kPerVec;    // lanes whose vectors share a bitmask word
+    constexpr int kWordsPerPass = 32 / kLanesPerWord;
+    constexpr bool kWiden = sizeof(OutT) > sizeof(TabT);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t dead = p.dead;
-    const uint32_t d32 = sizeof(OutT) == 2 ? (dead | (dead << 16)) : dead;
+    const uint32_t d32 = sizeof(TabT) == 2 ? (dead | (dead << 16)) : dead;
     const uint4 dead16 = make_uint4(d32, d32, d32, d32);
-    constexpr int kVec = 16 / sizeof(OutT);          // elements per 16-byte vector
-    constexpr int kVecPerLane = kSlice / kVec / 32;  // 2 (int32) or 1 (uint16)
-    // a slice is a whole number of 16-byte vectors, so every slice of an aligned row is aligned
-    const bool vec_ok = HAS_OUT && (reinterpret_cast<uintptr_t>(nrow) & 15) == 0;
-    const int eos_slice =
-        (p.eos_id >= 0 && q != p.dead && p.accept[q]) ? (p.eos_id >> kSliceShift) : -1;
-    const int last_full = p.N >> kSliceShift;  // slices below this index are complete
-    const typename E::type* lst = sink.lists + static_cast<size_t>(warp) * kSlice;
-    OutT* dst = HAS_OUT ? nrow + warp * kSlice : nullptr;
-    uint32_t* mdst = mrow + warp * kSliceWords;
+    // slices are multiples of 32 bytes of output, so an aligned row has aligned slices
+    const bool vec_ok = HAS_OUT && (reinterpret_cast<uintptr_t>(nrow) & (kWiden ? 31 : 15)) == 0;
+    const int eos_slice = (p.eos_id >= 0 && q != p.dead && p.accept[q]) ? (p.eos_id >> kShift) : -1;
+    const int last_full = p.N >> kShift;  // slices below this index are complete
+    const typename E::type* lst = sink.lists + static_cast<size_t>(warp) * kTok;
+    OutT* dst = HAS_OUT ? nrow + warp * kTok : nullptr;
+    uint32_t* mdst = mrow + warp * (kTok / 32);
     uint4* stage4 = reinterpret_cast<uint4*>(stage);
     // The first 32 survivors of a slice are fetched one slice ahead, so that the trip to
     // the L2-resident scratch overlaps the assembly of the previous slice.
@@ -287,53 +299,69 @@ __device__ __forceinline__ void assemble_row(const WalkParams& p, const Survivor
         const int next = sl + kWalkWarps;
         const int cnt_next = next < nslices ? sink.counts[next] : 0;
         typename E::type e_next = 0;
-        if (lane < cnt_next) e_next = lst[static_cast<size_t>(kWalkWarps) * kSlice + lane];
-        if (HAS_OUT) {
-#pragma unroll
-            for (int k = 0; k < kVecPerLane; ++k) stage4[lane + 32 * k] = dead16;
-        }
-        if (lane < kSliceWords) mwords[lane] = 0;
+        if (lane < cnt_next) e_next = lst[static_cast<size_t>(kWalkWarps) * kTok + lane];
+        stage4[lane] = dead16;
+        stage4[lane + 32] = dead16;
         __syncwarp();
-        if (lane < cnt) {
-            const uint32_t lid = E::lid(e0);
-            if (HAS_OUT) stage[lid] = static_cast<OutT>(E::state(e0));
-            atomicOr(&mwords[lid >> 5], 1u << (lid & 31));
-        }
+        if (lane < cnt) stage[E::lid(e0)] = static_cast<TabT>(E::state(e0));
         for (int i = 32 + lane; i < cnt; i += 32) {
             const typename E::type e = lst[i];
-            const uint32_t lid = E::lid(e);
-            if (HAS_OUT) stage[lid] = static_cast<OutT>(E::state(e));
-            atomicOr(&mwords[lid >> 5], 1u << (lid & 31));
+            stage[E::lid(e)] = static_cast<TabT>(E::state(e));
         }
-        if (sl == eos_slice && lane == 0) {
-            const int e = p.eos_id & (kSlice - 1);
-            if (HAS_OUT) stage[e] = static_cast<OutT>(q);
-            atomicOr(&mwords[e >> 5], 1u << (e & 31));
-        }
+        if (sl == eos_slice && lane == 0) stage[p.eos_id & (kTok - 1)] = static_cast<TabT>(q);
         __syncwarp();
-        if (sl < last_full) {
-            if (lane < kSliceWords) mdst[lane] = mwords[lane];
-            if (HAS_OUT) {
-                if (vec_ok) {
+        if (sl < last_full && (vec_ok || !HAS_OUT)) {
 #pragma unroll
-                    for (int k = 0; k < kVecPerLane; ++k)
-                        reinterpret_cast<uint4*>(dst)[lane + 32 * k] = stage4[lane + 32 * k];
-                } else {  // unaligned row: element-wise, still coalesced
-                    for (int i = lane; i < kSlice; i += 32) dst[i] = stage[i];
+            for (int k = 0; k < 2; ++k) {
+                const uint4 v = stage4[lane + 32 * k];
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                uint32_t bits = 0;  // one bit per state of this vector
+                if (sizeof(TabT) == 2) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        bits |= ((w[i] & 0xFFFFu) != dead ? 1u : 0u) << (2 * i);
+                        bits |= ((w[i] >> 16) != dead ? 1u : 0u) << (2 * i + 1);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) bits |= (w[i] != dead ? 1u : 0u) << i;
+                }
+                uint32_t word = bits << (kPerVec * (lane & (kLanesPerWord - 1)));
+#pragma unroll
+                for (int off = 1; off < kLanesPerWord; off <<= 1)
+                    word |= __shfl_xor_sync(kFullWarp, word, off);
+                if ((lane & (kLanesPerWord - 1)) == 0)
+                    mdst[k * kWordsPerPass + lane / kLanesPerWord] = word;
+                if (HAS_OUT) {
+                    if (kWiden) {  // 8 uint16 states -> 8 int32 states, one 32-byte store
+                        Vec32B o;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            o.w[2 * i] = w[i] & 0xFFFFu;
+                            o.w[2 * i + 1] = w[i] >> 16;
+                        }
+                        stg_32B(reinterpret_cast<uint8_t*>(dst) + (lane + 32 * k) * 32, o);
+                    } else {
+                        reinterpret_cast<uint4*>(dst)[lane + 32 * k] = v;
+                    }
                 }
             }
-        } else {  // ragged last slice
-            const int n = p.N - (sl << kSliceShift);
-            if (lane < (n + 31) / 32) mdst[lane] = mwords[lane];
-            if (HAS_OUT)
-                for (int i = lane; i < n; i += 32) dst[i] = stage[i];
+        } else {  // ragged last slice or unaligned row: element-wise, still coalesced
+            const int n = min(kTok, p.N - (sl << kShift));
+            for (int i0 = 0; i0 < n; i0 += 32) {
+                const int i = i0 + lane;
+                const uint32_t sv = i < n ? static_cast<uint32_t>(stage[i]) : dead;
+                const uint32_t word = __ballot_sync(kFullWarp, sv != dead);
+                if (lane == 0) mdst[i0 >> 5] = word;
+                if (HAS_OUT && i < n) dst[i] = static_cast<OutT>(sv);
+            }
         }
         __syncwarp();  // staging is refilled by the next slice
         cnt = cnt_next;
         e0 = e_next;
-        lst += static_cast<size_t>(kWalkWarps) * kSlice;
-        if (HAS_OUT) dst += kWalkWarps * kSlice;
-        mdst += kWalkWarps * kSliceWords;
+        lst += static_cast<size_t>(kWalkWarps) * kTok;
+        if (HAS_OUT) dst += kWalkWarps * kTok;
+        mdst += kWalkWarps * (kTok / 32);
     }
 }
 
@@ -382,15 +410,13 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
         raw_rows<OutT, HAS_OUT>(p);
         return;
     }
-    const int nslices = (p.N + kSlice - 1) >> kSliceShift;
-    // dynamic shared memory: per-warp staging, per-warp bitmask words, slice counters, table
-    constexpr size_t kStageBytes = HAS_OUT ? kSlice * sizeof(OutT) : 0;
+    constexpr int kTok = Slice<TabT>::kTokens;
+    const int nslices = (p.N + kTok - 1) >> Slice<TabT>::kShift;
+    // dynamic shared memory: per-warp staging, slice counters, chunk descriptors, table
     const int warp = threadIdx.x >> 5;
-    OutT* stage = reinterpret_cast<OutT*>(smem_raw + warp * kStageBytes);
-    uint32_t* mwords = reinterpret_cast<uint32_t*>(smem_raw + kWalkWarps * kStageBytes) + warp * kSliceWords;
-    int* counts = reinterpret_cast<int*>(smem_raw + kWalkWarps * (kStageBytes + kSliceWords * 4));
-    const size_t desc_off = (kWalkWarps * (kStageBytes + kSliceWords * 4) +
-                             static_cast<size_t>(nslices) * 4 + 15) / 16 * 16;
+    TabT* stage = reinterpret_cast<TabT*>(smem_raw + warp * kStageBytes);
+    int* counts = reinterpret_cast<int*>(smem_raw + kWalkWarps * kStageBytes);
+    const size_t desc_off = (kWalkWarps * kStageBytes + static_cast<size_t>(nslices) * 4 + 15) / 16 * 16;
     typename Desc<TabT>::type* descs = reinterpret_cast<typename Desc<TabT>::type*>(smem_raw + desc_off);
     const size_t table_off = (desc_off + kDescCap * sizeof(typename Desc<TabT>::type) + 127) / 128 * 128;
     TabT* stab = reinterpret_cast<TabT*>(smem_raw + table_off);
@@ -424,7 +450,7 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
         }
     }
     SurvivorSink<TabT> sink;
-    sink.lists = scratch + static_cast<size_t>(blockIdx.x) * nslices * kSlice;
+    sink.lists = scratch + static_cast<size_t>(blockIdx.x) * nslices * kTok;
     sink.counts = counts;
     sink.descs = descs;
     sink.desc_cap = kDescCap;
@@ -460,34 +486,28 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
                 walk_row<TabT, false, false>(p, gtab, C, Cs, two_level, s_gstart, sink, q);
         }
         __syncthreads();  // every survivor of the row is in its list (stores visible CTA-wide)
-        assemble_row<TabT, OutT, HAS_OUT>(p, sink, stage, mwords, nslices, q, nrow, mrow);
+        assemble_row<TabT, OutT, HAS_OUT>(p, sink, stage, nslices, q, nrow, mrow);
         __syncthreads();  // counters and lists are reused by the next row
     }
 }
 
-// Shared-memory bytes of walk_sparse besides the table.
-template <typename OutT, bool HAS_OUT>
-size_t sparse_fixed_smem(int32_t N) {
-    const size_t nslices = (static_cast<size_t>(N) + kSlice - 1) >> kSliceShift;
-    const size_t stage = HAS_OUT ? kSlice * sizeof(OutT) : 0;
-    const size_t desc_off = (kWalkWarps * (stage + kSliceWords * 4) + nslices * 4 + 15) / 16 * 16;
-    return (desc_off + kDescCap * 16 + 127) / 128 * 128;  // 16 = the larger descriptor type
+// Shared-memory bytes of walk_sparse in front of the table.
+template <typename TabT>
+size_t sparse_table_offset(int32_t N) {
+    const size_t nslices = (static_cast<size_t>(N) + Slice<TabT>::kTokens - 1) >> Slice<TabT>::kShift;
+    const size_t desc_off = (kWalkWarps * kStageBytes + nslices * 4 + 15) / 16 * 16;
+    return (desc_off + kDescCap * sizeof(typename Desc<TabT>::type) + 127) / 128 * 128;
 }
 
 template <typename TabT, typename OutT, bool HAS_OUT>
 cudaError_t launch_sparse(const WalkParams& p, void* scratch, int grid, cudaStream_t stream) {
     auto kernel = walk_sparse<TabT, OutT, HAS_OUT>;
-    const size_t fixed = sparse_fixed_smem<OutT, HAS_OUT>(p.N);
-    if (fixed + 1024 > p.smem_cap) return cudaErrorInvalidValue;
+    const size_t table_off = sparse_table_offset<TabT>(p.N);
+    if (table_off + 1024 > p.smem_cap) return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(p.smem_cap));
     if (e != cudaSuccess) return e;
     // what is left after staging, counters and the descriptor list may hold the table
-    const size_t nslices = (static_cast<size_t>(p.N) + kSlice - 1) >> kSliceShift;
-    const size_t stage = HAS_OUT ? kSlice * sizeof(OutT) : 0;
-    const size_t desc_off = (kWalkWarps * (stage + kSliceWords * 4) + nslices * 4 + 15) / 16 * 16;
-    const size_t table_off =
-        (desc_off + kDescCap * sizeof(typename Desc<TabT>::type) + 127) / 128 * 128;
     kernel<<<grid, kWalkThreads, p.smem_cap, stream>>>(
         p, static_cast<typename Entry<TabT>::type*>(scratch),
         static_cast<uint32_t>(p.smem_cap - table_off));
