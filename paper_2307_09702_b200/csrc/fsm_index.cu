@@ -62,7 +62,11 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     int cap = dev.smem_optin - 2048;  // static shared memory and alignment slack
     if (tune.smem_table_cap > 0 && tune.smem_table_cap < cap) cap = tune.smem_table_cap;
     // The sparse walk needs the survivor scratch and room for its per-warp staging.
-    const bool sparse = tune.walk_algo != 1 && !dense_only &&
+    // Automatic choice: the sparse walk works row by row, one CTA per row at a time, so it
+    // needs at least one row per SM to fill the device; small automata take the dense walk.
+    const bool want_sparse =
+        tune.walk_algo == 2 || (tune.walk_algo == 0 && q_end - q_begin >= dev.sm_count);
+    const bool sparse = want_sparse && !dense_only &&
                         (N + 255) / 256 <= kMaxSlices &&
                         sparse_table_offset<int32_t>(N) + 4096 <= static_cast<size_t>(dev.smem_optin - 2048);
 

@@ -6,19 +6,21 @@
 // SM works on one index row (one state q) at a time; the compressed table is staged in
 // shared memory once (bulk async copy) when it fits, else lookups use the read-only cache.
 //
-//   walk      only buckets whose key q can read are visited.  A unit of work is
-//             (readable first class, block of 32 second keys); warps take units from a
-//             shared counter.  Inside a bucket, lane = token, 32 tokens at a time,
-//             starting at the first byte the bucket key does not cover.  A surviving
-//             token appends (id within slice, end state) to the list of its *slice*
-//             (kSlice consecutive token ids).  The lists live in a per-CTA scratch in
-//             global memory that stays L2 resident; a list can hold a whole slice, so
-//             nothing can overflow.
+//   enumerate warps take units (readable first class, block of 32 second keys) from a
+//             shared counter; one lookup per key tells whether the bucket is readable;
+//             readable buckets are cut into 32-token chunk descriptors in shared memory.
+//   walk      warps pull chunks from the list; lane = token, starting at the first byte
+//             the bucket key does not cover.  A surviving token appends (id within slice,
+//             end state) to the list of its *slice* (1 KB of table-width states: 512
+//             consecutive token ids with 16-bit table entries).  The lists live in a
+//             per-CTA scratch in global memory that stays L2 resident; a list can hold a
+//             whole slice, so nothing can overflow.
 //   assemble  each warp takes slices in turn: it fills a 1 KB staging buffer in shared
-//             memory with `dead`, writes the slice's survivors into it, and stores the
-//             finished slice of the next-state row and its bitmask words with coalesced
-//             16-byte stores.  Global memory only sees full, write-once traffic for the
-//             outputs: the tokens whose first byte q cannot read cost no lookup at all.
+//             memory with `dead`, writes the slice's survivors into it, reads it back,
+//             derives the bitmask words from "state != dead" and stores the finished
+//             slice of the next-state row with coalesced 16- or 32-byte stores.  Global
+//             memory only sees full, write-once traffic for the outputs: the tokens
+//             whose first byte q cannot read cost no lookup at all.
 //
 // Three CTA barriers per row.  Results are identical to the dense walk.
 #pragma once
@@ -236,8 +238,10 @@ __device__ __forceinline__ void walk_row(const WalkParams& p, const TabT* __rest
     }
 }
 
-// Walks the chunks of the descriptor list; a warp takes two at a time and issues the
-// loads of both before walking either.
+// Walks the chunks of the descriptor list; a warp takes kPull at a time and issues the
+// loads of all of them before walking any.
+constexpr int kPull = 2;
+
 template <typename TabT, bool FULL>
 __device__ __forceinline__ void walk_chunks(const WalkParams& p, const TabT* __restrict__ tab,
                                             uint32_t Cs, const SurvivorSink<TabT>& sink) {
@@ -246,19 +250,23 @@ __device__ __forceinline__ void walk_chunks(const WalkParams& p, const TabT* __r
     const int total = sink.ctrs[1];
     while (true) {
         int i = 0;
-        if (lane == 0) i = atomicAdd(&sink.ctrs[2], 2);
+        if (lane == 0) i = atomicAdd(&sink.ctrs[2], kPull);
         i = __shfl_sync(kFullWarp, i, 0);
         if (i >= total) break;
-        const typename D::type d0 = sink.descs[i];
-        const bool two = i + 1 < total;
-        const typename D::type d1 = sink.descs[two ? i + 1 : i];
-        uint4 rec0, rec1;
-        int32_t id0, id1;
-        chunk_load(p, D::start(d0), D::count(d0), lane, rec0, id0);
-        chunk_load(p, D::start(d1), two ? D::count(d1) : 0, lane, rec1, id1);
-        chunk_finish_depth<TabT, FULL>(p, tab, Cs, sink, rec0, id0, D::state(d0), D::depth(d0));
-        if (two)
-            chunk_finish_depth<TabT, FULL>(p, tab, Cs, sink, rec1, id1, D::state(d1), D::depth(d1));
+        typename D::type d[kPull];
+        uint4 rec[kPull];
+        int32_t id[kPull];
+#pragma unroll
+        for (int k = 0; k < kPull; ++k) {
+            const bool have = i + k < total;
+            d[k] = sink.descs[have ? i + k : i];
+            chunk_load(p, D::start(d[k]), have ? D::count(d[k]) : 0, lane, rec[k], id[k]);
+        }
+#pragma unroll
+        for (int k = 0; k < kPull; ++k)
+            if (i + k < total)
+                chunk_finish_depth<TabT, FULL>(p, tab, Cs, sink, rec[k], id[k], D::state(d[k]),
+                                               D::depth(d[k]));
     }
 }
 
