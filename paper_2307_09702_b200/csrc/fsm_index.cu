@@ -73,7 +73,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     const int hash_blocks = Q < kHashBlocks ? Q : kHashBlocks;
     hash_columns<<<hash_blocks, 256 * kHashRowLanes, 0, stream>>>(
         dfa_trans, Q, dead_state, ws.partial, tune.weak_hash, ws.gcount, ws.count2, ws.cursor2,
-        status_word);
+        ws.row_ctr, status_word);
     derive_classes<<<1, 256, 0, stream>>>(ws.partial, hash_blocks, ws.meta, ws.cls, ws.class_rep);
     const int row_blocks = Q < 2 * dev.sm_count ? Q : 2 * dev.sm_count;
     const int tok_blocks = (G * 32 + 255) / 256;
@@ -119,6 +119,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     p.gstart = ws.gstart;
     p.count2 = ws.count2;
     p.start2 = ws.start2;
+    p.row_ctr = ws.row_ctr;
     p.mask = allowed_mask;
     p.next = next_state;
     p.status = status_word;

@@ -39,6 +39,7 @@ struct Workspace {
     int32_t* sid;        // [N] token id, same order as srec
     int32_t* gcount;     // [256] tokens per first-byte class
     int32_t* gstart;     // [257] first sorted position of each first-byte class
+    int32_t* row_ctr;    // [1] rows handed out by the sparse walk beyond the first one per CTA
     int32_t* count2;     // [kKeys] tokens per (first class, second key)
     int32_t* cursor2;    // [kKeys] placement cursors
     int32_t* start2;     // [kKeys] first sorted position of each (first class, second key)
@@ -74,6 +75,7 @@ inline Workspace carve(void* base, int32_t Q, int32_t N) {
     w.sid = reinterpret_cast<int32_t*>(tokens ? tokens + srec_bytes : nullptr);
     w.gcount = reinterpret_cast<int32_t*>(take(256 * sizeof(int32_t)));
     w.gstart = reinterpret_cast<int32_t*>(take(257 * sizeof(int32_t)));
+    w.row_ctr = reinterpret_cast<int32_t*>(take(sizeof(int32_t)));
     w.count2 = reinterpret_cast<int32_t*>(take(kKeys * sizeof(int32_t)));
     w.cursor2 = reinterpret_cast<int32_t*>(take(kKeys * sizeof(int32_t)));
     w.start2 = reinterpret_cast<int32_t*>(take(kKeys * sizeof(int32_t)));
@@ -104,6 +106,7 @@ struct WalkParams {
     const int32_t* gstart;
     const int32_t* count2;
     const int32_t* start2;
+    int32_t* row_ctr;
     // outputs
     uint32_t* mask;
     void* next;

@@ -16,7 +16,9 @@ constexpr int kHashRowLanes = 4;
 __global__ void __launch_bounds__(256 * kHashRowLanes)
 hash_columns(const int32_t* __restrict__ trans, int32_t Q, int32_t dead,
              uint64_t* __restrict__ partial, int weak, int32_t* __restrict__ gcount,
-             int32_t* __restrict__ count2, int32_t* __restrict__ cursor2, int32_t* status) {
+             int32_t* __restrict__ count2, int32_t* __restrict__ cursor2,
+             int32_t* __restrict__ row_ctr, int32_t* status) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) *row_ctr = 0;
     __shared__ uint64_t part[kHashRowLanes][256];
     const int b = threadIdx.x & 255, rl = threadIdx.x >> 8;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < kKeys; i += gridDim.x * blockDim.x) {

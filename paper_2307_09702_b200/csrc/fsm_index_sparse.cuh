@@ -413,6 +413,7 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
     __shared__ uint64_t bar;
     __shared__ int32_t s_gstart[260];
     __shared__ int s_ctrs[4];
+    __shared__ int s_next_row;
 
     if (p.meta->any_bad != 0) {
         raw_rows<OutT, HAS_OUT>(p);
@@ -464,14 +465,19 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
     sink.desc_cap = kDescCap;
     sink.ctrs = s_ctrs;
 
+    // Rows differ in cost (a state that reads the class of the space byte has three times
+    // the survivors), so after its first row a CTA takes rows from a global counter.
     const int nrows = p.q_end - p.q_begin;
-    for (int r = blockIdx.x; r < nrows; r += gridDim.x) {
+    int r = blockIdx.x;
+    while (r < nrows) {
         const int q = p.q_begin + r;
         OutT* nrow = HAS_OUT ? static_cast<OutT*>(p.next) + static_cast<size_t>(r) * p.N : nullptr;
         uint32_t* mrow = p.mask + static_cast<size_t>(r) * p.G;
         for (int i = threadIdx.x; i < nslices; i += kWalkThreads) counts[i] = 0;
         if (threadIdx.x < 4) s_ctrs[threadIdx.x] = 0;
+        if (threadIdx.x == 0) s_next_row = gridDim.x + atomicAdd(p.row_ctr, 1);
         __syncthreads();
+        const int next_row = s_next_row;
         if (full)
             walk_row<TabT, true, true>(p, stab, C, Cs, two_level, s_gstart, sink, q);
         else
@@ -496,6 +502,7 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
         __syncthreads();  // every survivor of the row is in its list (stores visible CTA-wide)
         assemble_row<TabT, OutT, HAS_OUT>(p, sink, stage, nslices, q, nrow, mrow);
         __syncthreads();  // counters and lists are reused by the next row
+        r = next_row;
     }
 }
 
