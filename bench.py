@@ -431,7 +431,7 @@ def run_ours(args):
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "note": "host DFA, vocabulary, logits and states copied in, tokens/states/finished "
                         "copied out, every step; the index stays on the device for its consumer"},
-        "gpu_launches": 7 * args.steps,
+        "gpu_launches": 8 * args.steps,
     }
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(w, starts)

@@ -7,7 +7,8 @@
 //   3. prepare_inputs  class-compressed table [Q x Cs] with exact verification that every
 //                      byte's column equals its class representative's column; token
 //                      records (dense walk) or bucket counts (sparse walk)
-//   3b. scan_keys, sort_tokens   sparse walk only: tokens sorted by (first, second) byte class
+//   3b. count_keys, scan_keys, sort_tokens   sparse walk only: tokens sorted by (first,
+//                      second) byte class
 //   4. walk            dense: every (state, token) pair walked by warp tiles;
 //      walk_sparse     only tokens of readable buckets walked, rows pre-filled with dead
 // If verification in 3 fails (a 64-bit hash collision) the walk reads the uncompressed
@@ -75,25 +76,34 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
         dfa_trans, Q, dead_state, ws.partial, tune.weak_hash, ws.gcount, ws.count2, ws.cursor2,
         ws.row_ctr, status_word);
     derive_classes<<<1, 256, 0, stream>>>(ws.partial, hash_blocks, ws.meta, ws.cls, ws.class_rep);
-    const int row_blocks = Q < 2 * dev.sm_count ? Q : 2 * dev.sm_count;
-    const int tok_blocks = (G * 32 + 255) / 256;
-    int32_t* count_into = sparse ? ws.count2 : nullptr;
+    const int row_blocks = Q < 16 * dev.sm_count ? Q : 16 * dev.sm_count;
+    const int tok_blocks = sparse ? 0 : (G * 32 + 255) / 256;  // dense walk: token records
     if (wide)
         prepare_inputs<int32_t><<<row_blocks + tok_blocks, 256, 0, stream>>>(
             dfa_trans, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
             row_blocks, ws.meta, ws.cls, ws.class_rep, static_cast<int32_t*>(ws.table),
-            ws.tok_cls, ws.tok_len, ws.gcount, count_into, status_word);
+            ws.tok_cls, ws.tok_len, status_word);
     else
         prepare_inputs<uint16_t><<<row_blocks + tok_blocks, 256, 0, stream>>>(
             dfa_trans, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
             row_blocks, ws.meta, ws.cls, ws.class_rep, static_cast<uint16_t*>(ws.table),
-            ws.tok_cls, ws.tok_len, ws.gcount, count_into, status_word);
+            ws.tok_cls, ws.tok_len, status_word);
     if (sparse) {
+        const int sort_blocks = (N + kSortTokens - 1) / kSortTokens;
+        const size_t key_smem = kKeys * sizeof(int);
+        if (cudaFuncSetAttribute(count_keys, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(key_smem)) != cudaSuccess ||
+            cudaFuncSetAttribute(sort_tokens, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(key_smem)) != cudaSuccess)
+            return FSM_ERR_CUDA;
+        count_keys<<<sort_blocks, kSortThreads, key_smem, stream>>>(
+            vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, ws.meta, ws.cls, ws.gcount,
+            ws.count2, status_word);
         scan_keys<<<kTwoLevelMaxC + 1, 256, 0, stream>>>(ws.meta, ws.gcount, ws.count2, ws.gstart,
                                                          ws.start2);
-        sort_tokens<<<(N + 255) / 256, 256, 0, stream>>>(vocab_bytes, vocab_offsets, vocab_nbytes,
-                                                         N, eos_id, ws.meta, ws.cls, ws.start2,
-                                                         ws.cursor2, ws.srec, ws.sid);
+        sort_tokens<<<sort_blocks, kSortThreads, key_smem, stream>>>(
+            vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, ws.meta, ws.cls, ws.start2,
+            ws.cursor2, ws.srec, ws.sid);
     }
     if (cudaGetLastError() != cudaSuccess) return FSM_ERR_CUDA;
 

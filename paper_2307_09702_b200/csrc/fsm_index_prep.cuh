@@ -100,10 +100,10 @@ __global__ void __launch_bounds__(256) derive_classes(const uint64_t* __restrict
 }
 
 // ---------------------------------------------------------------------------- 3
-// Blocks [0, row_blocks) compress and verify table rows; the remaining blocks work on
-// tokens: class records in token order for the dense walk (count2 == nullptr), or
-// bucket counts for the sparse walk.  Column C of the compressed table (the null class)
-// and the padding columns lead to the dead state, as does the whole row of the dead state.
+// Blocks [0, row_blocks) compress and verify table rows; the remaining blocks write the
+// class records of the tokens in token order (dense walk; the launch for the sparse walk
+// has no such blocks).  Column C of the compressed table (the null class) and the padding
+// columns lead to the dead state, as does the whole row of the dead state.
 template <typename TabT>
 __global__ void __launch_bounds__(256)
 prepare_inputs(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab_bytes,
@@ -111,8 +111,7 @@ prepare_inputs(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vo
                int32_t N, int32_t dead, int32_t eos_id, int row_blocks, IndexMeta* meta,
                const uint8_t* __restrict__ cls, const uint8_t* __restrict__ class_rep,
                TabT* __restrict__ table, uint4* __restrict__ tok_cls,
-               uint8_t* __restrict__ tok_len, int32_t* __restrict__ gcount,
-               int32_t* __restrict__ count2, int32_t* status) {
+               uint8_t* __restrict__ tok_len, int32_t* status) {
     const int C = meta->C, Cs = meta->Cs;
     if (static_cast<int>(blockIdx.x) < row_blocks) {
         __shared__ int32_t row[256];
@@ -134,25 +133,6 @@ prepare_inputs(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vo
             atomicExch(&meta->any_bad, 1);
             raise_flag(status, FSM_FLAG_CLASS_SPLIT);
         }
-    } else if (count2 != nullptr) {
-        __shared__ int hist[256];
-        __shared__ uint8_t s_cls[256];
-        hist[threadIdx.x] = 0;
-        s_cls[threadIdx.x] = cls[threadIdx.x];
-        __syncthreads();
-        bool bad = false;
-        const bool two = meta->two_level != 0;
-        const int64_t v = static_cast<int64_t>(blockIdx.x - row_blocks) * 256 + threadIdx.x;
-        const TokenInfo t = token_info(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, s_cls, v, &bad);
-        // one atomic per distinct key of the warp
-        const int key = t.len > 0 ? bucket_key(two, t.first, t.second_key) : -1;
-        const uint32_t peers = __match_any_sync(kFullWarp, key);
-        if (t.len > 0) {
-            atomicAdd(&hist[t.first], 1);
-            if ((threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&count2[key], __popc(peers));
-        }
-        if (__syncthreads_or(bad) && threadIdx.x == 0) raise_flag(status, FSM_FLAG_OFFSETS);
-        if (hist[threadIdx.x] > 0) atomicAdd(&gcount[threadIdx.x], hist[threadIdx.x]);
     } else {
         const int64_t slots = (static_cast<int64_t>(N) + 31) / 32 * 32;
         const int64_t v = static_cast<int64_t>(blockIdx.x - row_blocks) * 256 + threadIdx.x;
@@ -167,8 +147,13 @@ prepare_inputs(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vo
                 len = static_cast<int>(min(o1 - o0, static_cast<int64_t>(kInlineBytes + 1)));
                 const int n = min(len, kInlineBytes);
                 if (n > 0) w[0] = 0;
-                for (int i = 0; i < n; ++i)
-                    w[i >> 2] |= static_cast<uint32_t>(cls[vocab_bytes[o0 + i]]) << ((i & 3) * 8);
+                uint8_t raw[kInlineBytes];
+#pragma unroll
+                for (int i = 0; i < kInlineBytes; ++i)  // independent loads, issued together
+                    raw[i] = i < n ? vocab_bytes[o0 + i] : 0;
+#pragma unroll
+                for (int i = 0; i < kInlineBytes; ++i)
+                    if (i < n) w[i >> 2] |= static_cast<uint32_t>(cls[raw[i]]) << ((i & 3) * 8);
             }
         }
         tok_cls[v] = make_uint4(w[0], w[1], w[2], w[3]);
@@ -180,8 +165,8 @@ prepare_inputs(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vo
 // Token order of the sparse walk: a counting sort by bucket key - the class of the
 // first byte and, when there are at most kTwoLevelMaxC classes, the class of the second
 // byte (key 0 = one-byte token).  scan_keys turns the counts into first positions
-// (block c0 handles the keys of first class c0); sort_tokens places 256 tokens per
-// block.  A record keeps the length and the classes of bytes 1..15; `sid` holds the
+// (block c0 handles the keys of first class c0); count_keys / sort_tokens handle 1,024
+// tokens per block.  A record keeps the length and the classes of bytes 1..15; `sid` holds the
 // token id.
 __global__ void __launch_bounds__(256)
 scan_keys(const IndexMeta* __restrict__ meta, const int32_t* __restrict__ gcount,
@@ -234,32 +219,78 @@ scan_keys(const IndexMeta* __restrict__ meta, const int32_t* __restrict__ gcount
     if (t <= C) start2[c0 * kKeyStride + t] = gst[c0] + before + incl - mine;
 }
 
-__global__ void __launch_bounds__(256)
+// Bucket keys are counted and ranked per block of kSortTokens tokens in shared memory
+// (one counter per key), so that global memory sees one atomic per block and key instead
+// of one per token: tokens that start with a space are a third of a BPE vocabulary and
+// would otherwise all hit the same few counters.
+constexpr int kSortThreads = 1024;
+constexpr int kSortTokens = kSortThreads;
+
+__global__ void __launch_bounds__(kSortThreads)
+count_keys(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vocab_offsets,
+           int64_t vocab_nbytes, int32_t N, int32_t eos_id, const IndexMeta* __restrict__ meta,
+           const uint8_t* __restrict__ cls, int32_t* __restrict__ gcount,
+           int32_t* __restrict__ count2, int32_t* status) {
+    extern __shared__ int s_cnt[];  // [kKeys]
+    __shared__ int hist[256];
+    __shared__ uint8_t s_cls[256];
+    if (threadIdx.x < 256) {
+        hist[threadIdx.x] = 0;
+        s_cls[threadIdx.x] = cls[threadIdx.x];
+    }
+    const bool two = meta->two_level != 0;
+    const int nkeys = two ? kKeys : 256;
+    for (int i = threadIdx.x; i < nkeys; i += kSortThreads) s_cnt[i] = 0;
+    __syncthreads();
+    bool bad = false;
+    const int64_t v = static_cast<int64_t>(blockIdx.x) * kSortTokens + threadIdx.x;
+    const TokenInfo t = token_info(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, s_cls, v, &bad);
+    if (t.len > 0) {
+        atomicAdd(&hist[t.first], 1);
+        atomicAdd(&s_cnt[bucket_key(two, t.first, t.second_key)], 1);
+    }
+    if (__syncthreads_or(bad) && threadIdx.x == 0) raise_flag(status, FSM_FLAG_OFFSETS);
+    for (int i = threadIdx.x; i < nkeys; i += kSortThreads)
+        if (s_cnt[i] > 0) atomicAdd(&count2[i], s_cnt[i]);
+    if (threadIdx.x < 256 && hist[threadIdx.x] > 0) atomicAdd(&gcount[threadIdx.x], hist[threadIdx.x]);
+}
+
+__global__ void __launch_bounds__(kSortThreads)
 sort_tokens(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vocab_offsets,
             int64_t vocab_nbytes, int32_t N, int32_t eos_id, const IndexMeta* __restrict__ meta,
             const uint8_t* __restrict__ cls, const int32_t* __restrict__ start2,
             int32_t* __restrict__ cursor2, uint4* __restrict__ srec, int32_t* __restrict__ sid) {
+    extern __shared__ int s_cnt[];  // [kKeys] count, then the block's base position per key
     __shared__ uint8_t s_cls[256];
-    s_cls[threadIdx.x] = cls[threadIdx.x];
-    __syncthreads();
+    if (threadIdx.x < 256) s_cls[threadIdx.x] = cls[threadIdx.x];
     const bool two = meta->two_level != 0;
+    const int nkeys = two ? kKeys : 256;
+    for (int i = threadIdx.x; i < nkeys; i += kSortThreads) s_cnt[i] = 0;
+    __syncthreads();
     bool bad = false;
-    const int64_t v = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
+    const int64_t v = static_cast<int64_t>(blockIdx.x) * kSortTokens + threadIdx.x;
     const TokenInfo t = token_info(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, s_cls, v, &bad);
-    // one cursor atomic per distinct key of the warp
-    const int key = t.len > 0 ? bucket_key(two, t.first, t.second_key) : -1;
-    const uint32_t peers = __match_any_sync(kFullWarp, key);
-    const int lane = threadIdx.x & 31;
-    const int leader = __ffs(peers) - 1;
-    int base = 0;
-    if (t.len > 0 && lane == leader) base = atomicAdd(&cursor2[key], __popc(peers));
-    base = __shfl_sync(kFullWarp, base, leader);
+    const int key = t.len > 0 ? bucket_key(two, t.first, t.second_key) : 0;
+    int rank = 0;
+    if (t.len > 0) rank = atomicAdd(&s_cnt[key], 1);
+    __syncthreads();
+    // one global atomic per key present in the block reserves its positions
+    for (int i = threadIdx.x; i < nkeys; i += kSortThreads) {
+        const int c = s_cnt[i];
+        if (c > 0) s_cnt[i] = start2[i] + atomicAdd(&cursor2[i], c);
+    }
+    __syncthreads();
     if (t.len > 0) {
-        const int pos = start2[key] + base + __popc(peers & ((1u << lane) - 1u));
+        const int pos = s_cnt[key] + rank;
         uint32_t w[4] = {static_cast<uint32_t>(t.len), 0, 0, 0};
         const int nb = min(t.len, kInlineBytes);
-        for (int i = 1; i < nb; ++i)
-            w[i >> 2] |= static_cast<uint32_t>(s_cls[vocab_bytes[t.start + i]]) << ((i & 3) * 8);
+        uint8_t raw[kInlineBytes];
+#pragma unroll
+        for (int i = 1; i < kInlineBytes; ++i)  // independent loads, issued together
+            raw[i] = i < nb ? vocab_bytes[t.start + i] : 0;
+#pragma unroll
+        for (int i = 1; i < kInlineBytes; ++i)
+            if (i < nb) w[i >> 2] |= static_cast<uint32_t>(s_cls[raw[i]]) << ((i & 3) * 8);
         srec[pos] = make_uint4(w[0], w[1], w[2], w[3]);
         sid[pos] = static_cast<int32_t>(v);
     }
