@@ -93,8 +93,11 @@ size_t fsm_index_workspace_bytes(int32_t Q, int32_t N, int64_t vocab_nbytes);
  *                  Aligned to its element size.
  *   state_dtype    FSM_STATE_I32, or FSM_STATE_U16 (requires Q <= 65535).
  *   workspace      device scratch, 256-byte aligned, at least
- *                  fsm_index_workspace_bytes(Q, N, vocab_nbytes) bytes.  Contents on
- *                  entry are irrelevant; concurrent calls need separate workspaces.
+ *                  fsm_index_workspace_bytes(Q, N, vocab_nbytes) bytes (the compressed
+ *                  table, the token records and, for the work-avoiding walk, per-CTA
+ *                  survivor lists of min(Q,160) * N entries: about 85 MB for 1,001
+ *                  states and 128,256 tokens).  Contents on entry are irrelevant;
+ *                  concurrent calls need separate workspaces.
  *   status_word    device int32 or NULL.
  *
  * fsm_index_build_rows builds only rows q_begin <= q < q_end, written to
