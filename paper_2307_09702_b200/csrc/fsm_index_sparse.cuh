@@ -38,6 +38,7 @@ template <typename TabT> struct Slice {
     static constexpr int kTokens = 1 << kShift;
 };
 constexpr int kMaxSliceTokens = 512;
+constexpr int kMaskWords = kMaxSliceTokens / 32;  // bitmask words of one slice
 constexpr int kMaxSlices = 8192;          // vocabularies up to 2 M tokens (else the dense walk)
 constexpr int kDescCap = 4096;            // chunk descriptors kept per row
 
@@ -272,19 +273,16 @@ __device__ __forceinline__ void walk_chunks(const WalkParams& p, const TabT* __r
 
 // Assembles and stores the slices of one row; warp w takes slices w, w+32, ...
 // The slice is staged in table-entry width (1 KB per warp): filled with `dead`, then
-// the survivors are written into it.  Each lane then reads back two 16-byte vectors,
-// derives their bitmask bits from "state != dead" (a warp reduce joins the lanes of a
-// word), widens the states if the output is wider than the table entries, and stores.
+// the survivors are written into it and OR their bits into the slice's bitmask words
+// (shared memory).  Each lane then reads back two 16-byte vectors, widens the states if
+// the output is wider than the table entries, and stores.
 template <typename TabT, typename OutT, bool HAS_OUT>
 __device__ __forceinline__ void assemble_row(const WalkParams& p, const SurvivorSink<TabT>& sink,
-                                             TabT* stage, int nslices, int q, OutT* nrow,
-                                             uint32_t* mrow) {
+                                             TabT* stage, uint32_t* mwords, int nslices, int q,
+                                             OutT* nrow, uint32_t* mrow) {
     using E = Entry<TabT>;
     constexpr int kTok = Slice<TabT>::kTokens;
     constexpr int kShift = Slice<TabT>::kShift;
-    constexpr int kPerVec = 16 / sizeof(TabT);     // states per 16-byte staging vector
-    constexpr int kLanesPerWord = 32 / kPerVec;    // lanes whose vectors share a bitmask word
-    constexpr int kWordsPerPass = 32 / kLanesPerWord;
     constexpr bool kWiden = sizeof(OutT) > sizeof(TabT);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t dead = p.dead;
@@ -310,38 +308,33 @@ __device__ __forceinline__ void assemble_row(const WalkParams& p, const Survivor
         if (lane < cnt_next) e_next = lst[static_cast<size_t>(kWalkWarps) * kTok + lane];
         stage4[lane] = dead16;
         stage4[lane + 32] = dead16;
+        if (lane < kTok / 32) mwords[lane] = 0;
         __syncwarp();
-        if (lane < cnt) stage[E::lid(e0)] = static_cast<TabT>(E::state(e0));
+        if (lane < cnt) {
+            const uint32_t lid = E::lid(e0);
+            stage[lid] = static_cast<TabT>(E::state(e0));
+            atomicOr(&mwords[lid >> 5], 1u << (lid & 31));
+        }
         for (int i = 32 + lane; i < cnt; i += 32) {
             const typename E::type e = lst[i];
-            stage[E::lid(e)] = static_cast<TabT>(E::state(e));
+            const uint32_t lid = E::lid(e);
+            stage[lid] = static_cast<TabT>(E::state(e));
+            atomicOr(&mwords[lid >> 5], 1u << (lid & 31));
         }
-        if (sl == eos_slice && lane == 0) stage[p.eos_id & (kTok - 1)] = static_cast<TabT>(q);
+        if (sl == eos_slice && lane == 0) {
+            const uint32_t lid = p.eos_id & (kTok - 1);
+            stage[lid] = static_cast<TabT>(q);
+            atomicOr(&mwords[lid >> 5], 1u << (lid & 31));
+        }
         __syncwarp();
         if (sl < last_full && (vec_ok || !HAS_OUT)) {
+            if (lane < kTok / 32) mdst[lane] = mwords[lane];
+            if (HAS_OUT) {
 #pragma unroll
-            for (int k = 0; k < 2; ++k) {
-                const uint4 v = stage4[lane + 32 * k];
-                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-                uint32_t bits = 0;  // one bit per state of this vector
-                if (sizeof(TabT) == 2) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        bits |= ((w[i] & 0xFFFFu) != dead ? 1u : 0u) << (2 * i);
-                        bits |= ((w[i] >> 16) != dead ? 1u : 0u) << (2 * i + 1);
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) bits |= (w[i] != dead ? 1u : 0u) << i;
-                }
-                uint32_t word = bits << (kPerVec * (lane & (kLanesPerWord - 1)));
-#pragma unroll
-                for (int off = 1; off < kLanesPerWord; off <<= 1)
-                    word |= __shfl_xor_sync(kFullWarp, word, off);
-                if ((lane & (kLanesPerWord - 1)) == 0)
-                    mdst[k * kWordsPerPass + lane / kLanesPerWord] = word;
-                if (HAS_OUT) {
+                for (int k = 0; k < 2; ++k) {
+                    const uint4 v = stage4[lane + 32 * k];
                     if (kWiden) {  // 8 uint16 states -> 8 int32 states, one 32-byte store
+                        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
                         Vec32B o;
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
@@ -424,8 +417,10 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
     // dynamic shared memory: per-warp staging, slice counters, chunk descriptors, table
     const int warp = threadIdx.x >> 5;
     TabT* stage = reinterpret_cast<TabT*>(smem_raw + warp * kStageBytes);
-    int* counts = reinterpret_cast<int*>(smem_raw + kWalkWarps * kStageBytes);
-    const size_t desc_off = (kWalkWarps * kStageBytes + static_cast<size_t>(nslices) * 4 + 15) / 16 * 16;
+    uint32_t* mwords = reinterpret_cast<uint32_t*>(smem_raw + kWalkWarps * kStageBytes) + warp * kMaskWords;
+    int* counts = reinterpret_cast<int*>(smem_raw + kWalkWarps * (kStageBytes + kMaskWords * 4));
+    const size_t desc_off = (kWalkWarps * (kStageBytes + kMaskWords * 4) +
+                             static_cast<size_t>(nslices) * 4 + 15) / 16 * 16;
     typename Desc<TabT>::type* descs = reinterpret_cast<typename Desc<TabT>::type*>(smem_raw + desc_off);
     const size_t table_off = (desc_off + kDescCap * sizeof(typename Desc<TabT>::type) + 127) / 128 * 128;
     TabT* stab = reinterpret_cast<TabT*>(smem_raw + table_off);
@@ -500,7 +495,7 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
                 walk_row<TabT, false, false>(p, gtab, C, Cs, two_level, s_gstart, sink, q);
         }
         __syncthreads();  // every survivor of the row is in its list (stores visible CTA-wide)
-        assemble_row<TabT, OutT, HAS_OUT>(p, sink, stage, nslices, q, nrow, mrow);
+        assemble_row<TabT, OutT, HAS_OUT>(p, sink, stage, mwords, nslices, q, nrow, mrow);
         __syncthreads();  // counters and lists are reused by the next row
         r = next_row;
     }
@@ -510,7 +505,7 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
 template <typename TabT>
 size_t sparse_table_offset(int32_t N) {
     const size_t nslices = (static_cast<size_t>(N) + Slice<TabT>::kTokens - 1) >> Slice<TabT>::kShift;
-    const size_t desc_off = (kWalkWarps * kStageBytes + nslices * 4 + 15) / 16 * 16;
+    const size_t desc_off = (kWalkWarps * (kStageBytes + kMaskWords * 4) + nslices * 4 + 15) / 16 * 16;
     return (desc_off + kDescCap * sizeof(typename Desc<TabT>::type) + 127) / 128 * 128;
 }
 
