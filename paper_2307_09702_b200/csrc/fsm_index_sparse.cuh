@@ -358,6 +358,7 @@ __device__ __forceinline__ void assemble_row(const WalkParams& p, const Survivor
             }
         }
         __syncwarp();  // staging is refilled by the next slice
+        if (lane == 0) sink.counts[sl] = 0;  // ready for the next row's survivors
         cnt = cnt_next;
         e0 = e_next;
         lst += static_cast<size_t>(kWalkWarps) * kTok;
@@ -405,8 +406,8 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
     extern __shared__ __align__(128) uint8_t smem_raw[];
     __shared__ uint64_t bar;
     __shared__ int32_t s_gstart[260];
-    __shared__ int s_ctrs[4];
-    __shared__ int s_next_row;
+    __shared__ int s_ctrs[8];      // two sets of row counters (see SurvivorSink::ctrs)
+    __shared__ int s_next_row[2];
 
     if (p.meta->any_bad != 0) {
         raw_rows<OutT, HAS_OUT>(p);
@@ -462,23 +463,37 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
 
     // Rows differ in cost (a state that reads the class of the space byte has three times
     // the survivors), so after its first row a CTA takes rows from a global counter.
+    //
+    // Per row: walk the chunk list | barrier | assemble the row, then enumerate the next
+    // row's chunks (no barrier in between: enumeration touches only the descriptor list
+    // and its counters, which nobody reads during assembly) | barrier.  The counters are
+    // double buffered by row parity; the slice counters are cleared by the warp that
+    // assembled the slice.
     const int nrows = p.q_end - p.q_begin;
-    int r = blockIdx.x;
+    auto enumerate = [&](int row, int par) {
+        SurvivorSink<TabT> s2 = sink;
+        s2.ctrs = s_ctrs + 4 * par;
+        if (full)
+            walk_row<TabT, true, true>(p, stab, C, Cs, two_level, s_gstart, s2, p.q_begin + row);
+        else
+            walk_row<TabT, false, true>(p, gtab, C, Cs, two_level, s_gstart, s2, p.q_begin + row);
+    };
+    for (int i = threadIdx.x; i < nslices; i += kWalkThreads) counts[i] = 0;
+    if (threadIdx.x < 8) s_ctrs[threadIdx.x] = 0;
+    __syncthreads();
+    int r = blockIdx.x, par = 0;
+    if (r < nrows) enumerate(r, par);
+    __syncthreads();  // the chunk list of the first row is complete
     while (r < nrows) {
         const int q = p.q_begin + r;
         OutT* nrow = HAS_OUT ? static_cast<OutT*>(p.next) + static_cast<size_t>(r) * p.N : nullptr;
         uint32_t* mrow = p.mask + static_cast<size_t>(r) * p.G;
-        for (int i = threadIdx.x; i < nslices; i += kWalkThreads) counts[i] = 0;
-        if (threadIdx.x < 4) s_ctrs[threadIdx.x] = 0;
-        if (threadIdx.x == 0) s_next_row = gridDim.x + atomicAdd(p.row_ctr, 1);
-        __syncthreads();
-        const int next_row = s_next_row;
-        if (full)
-            walk_row<TabT, true, true>(p, stab, C, Cs, two_level, s_gstart, sink, q);
-        else
-            walk_row<TabT, false, true>(p, gtab, C, Cs, two_level, s_gstart, sink, q);
-        __syncthreads();  // the chunk list of the row is complete
-        if (s_ctrs[3] == 0) {
+        sink.ctrs = s_ctrs + 4 * par;
+        if (threadIdx.x == 0) {  // next row and its counters, published by the barrier below
+            s_next_row[par ^ 1] = gridDim.x + atomicAdd(p.row_ctr, 1);
+            for (int i = 0; i < 4; ++i) s_ctrs[4 * (par ^ 1) + i] = 0;
+        }
+        if (sink.ctrs[3] == 0) {
             if (full)
                 walk_chunks<TabT, true>(p, stab, Cs, sink);
             else
@@ -487,7 +502,7 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
             // more chunks than the list holds (a state that reads almost everything):
             // walk the buckets unit by unit instead
             __syncthreads();
-            if (threadIdx.x == 0) s_ctrs[0] = 0;
+            if (threadIdx.x == 0) sink.ctrs[0] = 0;
             __syncthreads();
             if (full)
                 walk_row<TabT, true, false>(p, stab, C, Cs, two_level, s_gstart, sink, q);
@@ -495,9 +510,12 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
                 walk_row<TabT, false, false>(p, gtab, C, Cs, two_level, s_gstart, sink, q);
         }
         __syncthreads();  // every survivor of the row is in its list (stores visible CTA-wide)
+        const int next_row = s_next_row[par ^ 1];
         assemble_row<TabT, OutT, HAS_OUT>(p, sink, stage, mwords, nslices, q, nrow, mrow);
-        __syncthreads();  // counters and lists are reused by the next row
+        if (next_row < nrows) enumerate(next_row, par ^ 1);
+        __syncthreads();  // slice counters cleared, next chunk list complete
         r = next_row;
+        par ^= 1;
     }
 }
 
