@@ -17,6 +17,7 @@
 #include "fsm_index_dense.cuh"
 #include "fsm_index_prep.cuh"
 #include "fsm_index_sparse.cuh"
+#include "fsm_index_bucket.cuh"
 
 extern "C" size_t fsm_index_workspace_bytes(int32_t Q, int32_t N, int64_t vocab_nbytes) {
     if (Q <= 0 || N <= 0 || vocab_nbytes < 0) return 0;
@@ -67,7 +68,10 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     // needs at least one row per SM to fill the device; small automata take the dense walk.
     const bool want_sparse =
         tune.walk_algo == 2 || (tune.walk_algo == 0 && q_end - q_begin >= dev.sm_count);
-    const bool sparse = want_sparse && !dense_only &&
+    // Bitmask-only builds take the bucket walk (no dense rows to assemble).
+    const bool bucket = next_state == nullptr && !dense_only &&
+                        (tune.walk_algo == 3 || tune.walk_algo == 0);
+    const bool sparse = (bucket || want_sparse) && !dense_only &&
                         (N + 255) / 256 <= kMaxSlices &&
                         sparse_table_offset<int32_t>(N) + 4096 <= static_cast<size_t>(dev.smem_optin - 2048);
 
@@ -78,16 +82,18 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     derive_classes<<<1, 256, 0, stream>>>(ws.partial, hash_blocks, ws.meta, ws.cls, ws.class_rep);
     const int row_blocks = Q < 16 * dev.sm_count ? Q : 16 * dev.sm_count;
     const int tok_blocks = sparse ? 0 : (G * 32 + 255) / 256;  // dense walk: token records
+    uint32_t* live = bucket ? ws.live : nullptr;
+    uint32_t* planes = bucket ? ws.planes : nullptr;
     if (wide)
         prepare_inputs<int32_t><<<row_blocks + tok_blocks, 256, 0, stream>>>(
             dfa_trans, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
             row_blocks, ws.meta, ws.cls, ws.class_rep, static_cast<int32_t*>(ws.table),
-            ws.tok_cls, ws.tok_len, status_word);
+            ws.tok_cls, ws.tok_len, live, status_word);
     else
         prepare_inputs<uint16_t><<<row_blocks + tok_blocks, 256, 0, stream>>>(
             dfa_trans, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
             row_blocks, ws.meta, ws.cls, ws.class_rep, static_cast<uint16_t*>(ws.table),
-            ws.tok_cls, ws.tok_len, status_word);
+            ws.tok_cls, ws.tok_len, live, status_word);
     if (sparse) {
         const int sort_blocks = (N + kSortTokens - 1) / kSortTokens;
         const size_t key_smem = kKeys * sizeof(int);
@@ -98,7 +104,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
             return FSM_ERR_CUDA;
         count_keys<<<sort_blocks, kSortThreads, key_smem, stream>>>(
             vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, ws.meta, ws.cls, ws.gcount,
-            ws.count2, status_word);
+            ws.count2, planes, status_word);
         scan_keys<<<kTwoLevelMaxC + 1, 256, 0, stream>>>(ws.meta, ws.gcount, ws.count2, ws.gstart,
                                                          ws.start2);
         sort_tokens<<<sort_blocks, kSortThreads, key_smem, stream>>>(
@@ -126,6 +132,8 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     p.tok_len = ws.tok_len;
     p.srec = ws.srec;
     p.sid = ws.sid;
+    p.planes = ws.planes;
+    p.live = ws.live;
     p.gstart = ws.gstart;
     p.count2 = ws.count2;
     p.start2 = ws.start2;
@@ -150,7 +158,10 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     if (tune.walk_ctas > 0 && tune.walk_ctas < grid) grid = tune.walk_ctas;
     const int prof = profile_begin(stream);
     cudaError_t e;
-    if (sparse)
+    if (bucket)
+        e = wide ? launch_bucket<int32_t>(p, dev.sm_count, stream)
+                 : launch_bucket<uint16_t>(p, dev.sm_count, stream);
+    else if (sparse)
         e = wide ? launch_sparse_for<int32_t>(p, ws.survivors, static_cast<int>(grid), state_dtype,
                                               next_state != nullptr, stream)
                  : launch_sparse_for<uint16_t>(p, ws.survivors, static_cast<int>(grid), state_dtype,

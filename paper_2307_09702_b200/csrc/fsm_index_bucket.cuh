@@ -1,0 +1,235 @@
+// Bucket walk of the index build for bitmask-only builds (no next-state table): two kernels
+// that never visit a (state, token) pair whose first two bytes the state cannot read.
+//
+//   mask_onebyte  A token of one byte is allowed in state q iff q reads the class of that
+//                 byte, so the bitmask words of all one-byte tokens are the OR, over the
+//                 classes q reads, of per-class bit planes prepared once per vocabulary.
+//                 The kernel writes every bitmask word (tokens of two or more bytes get
+//                 their bits from walk_buckets).
+//   walk_buckets  Tokens are kept sorted by (class of byte 0, class of byte 1).  A warp
+//                 takes 32 consecutive sorted tokens (lane = token, record in registers)
+//                 and a block of 128 states; for every key present in the window it scans
+//                 the states (lane = state, two table lookups) and walks the window from
+//                 each state that reads the key, starting at byte 2.  A surviving token
+//                 sets its bitmask bit with an atomic OR.
+//
+// The compressed table is staged in shared memory (bulk async copy) when it fits, else
+// lookups use the read-only cache.  Results are identical to the dense walk.
+#pragma once
+
+#include "fsm_index_common.cuh"
+#include "fsm_index_sparse.cuh"
+
+namespace fsm {
+namespace {
+
+constexpr int kStatesPerTask = 128;   // states scanned by one walk_buckets task
+
+// Stages the whole compressed table in shared memory when it fits.  Returns false (after
+// raising the flag) when the bounded wait gave up; `full` tells whether the table is in
+// shared memory.
+template <typename TabT>
+__device__ __forceinline__ bool stage_table(const WalkParams& p, TabT* stab, uint64_t* bar,
+                                            uint32_t table_cap, uint32_t Cs, bool& full) {
+    const uint64_t table_bytes = static_cast<uint64_t>(p.Q) * Cs * sizeof(TabT);
+    full = table_bytes <= table_cap;
+    if (!full) return true;
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const uint32_t bytes = static_cast<uint32_t>(table_bytes);
+        mbar_expect_tx(bar, bytes);
+        for (uint32_t o = 0; o < bytes; o += kBulkChunk)
+            bulk_copy_g2s(reinterpret_cast<uint8_t*>(stab) + o,
+                          reinterpret_cast<const uint8_t*>(p.table) + o, min(kBulkChunk, bytes - o),
+                          bar);
+    }
+    bool ok = mbar_wait_bounded(bar, 0);
+    if (!ok) ok = mbar_wait_bounded(bar, 0);  // drain before giving up
+    if (!__syncthreads_and(ok)) {
+        if (threadIdx.x == 0) raise_flag(p.status, FSM_FLAG_WAIT_TIMEOUT);
+        return false;
+    }
+    return true;
+}
+
+// ---------------------------------------------------------------------------------------
+// Bitmask words of the one-byte tokens (and zeros elsewhere).  Block (x, y): the 128
+// bitmask words 128x .. 128x+127 of the rows 8y + warp, 8y + warp + 8 gridDim.y, ...; those
+// words of the first 64 planes sit in shared memory; lane l handles words l, l+32, l+64,
+// l+96.
+constexpr int kObThreads = 256;
+constexpr int kObWords = 128;
+constexpr int kObSmemClasses = 64;  // planes of further classes are read through the cache
+
+__global__ void __launch_bounds__(kObThreads) mask_onebyte(const WalkParams p) {
+    __shared__ uint32_t s_pl[kObSmemClasses * kObWords];  // planes of the first classes
+    __shared__ uint8_t s_live[kObThreads / 32][256];      // classes read by the warp's row
+    if (p.meta->any_bad != 0) {
+        // exact fallback: every token walked through the uncompressed table
+        if (blockIdx.y == 0) raw_rows<int32_t, false>(p);
+        return;
+    }
+    const int C = p.meta->C;
+    const int nrows = p.q_end - p.q_begin;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int w0 = blockIdx.x * kObWords;
+    const int c_smem = min(C, kObSmemClasses);
+    for (int i = threadIdx.x; i < c_smem * kObWords; i += kObThreads) {
+        const int wd = w0 + (i & (kObWords - 1));
+        s_pl[i] = wd < p.G ? p.planes[static_cast<size_t>(i / kObWords) * p.G + wd] : 0;
+    }
+    __syncthreads();
+    const int eos_word = p.eos_id >= 0 ? (p.eos_id >> 5) - w0 : -1;
+    uint8_t* mine = s_live[warp];
+    for (int r = blockIdx.y * (kObThreads / 32) + warp; r < nrows; r += gridDim.y * (kObThreads / 32)) {
+        const int q = p.q_begin + r;
+        // the classes q reads, as a list
+        int nlive = 0;
+        for (int k = 0; k * 32 < C; ++k) {
+            const uint32_t m = __ldg(p.live + static_cast<size_t>(q) * 8 + k);
+            if ((m >> lane) & 1u) mine[nlive + __popc(m & ((1u << lane) - 1u))] = static_cast<uint8_t>(k * 32 + lane);
+            nlive += __popc(m);
+        }
+        __syncwarp();
+        uint32_t acc[kObWords / 32] = {0, 0, 0, 0};
+        for (int j = 0; j < nlive; ++j) {
+            const int c = mine[j];
+            if (c < kObSmemClasses) {
+                const uint32_t* pl = s_pl + c * kObWords + lane;
+#pragma unroll
+                for (int i = 0; i < kObWords / 32; ++i) acc[i] |= pl[32 * i];
+            } else {
+                const uint32_t* pl = p.planes + static_cast<size_t>(c) * p.G + w0 + lane;
+#pragma unroll
+                for (int i = 0; i < kObWords / 32; ++i)
+                    if (w0 + lane + 32 * i < p.G) acc[i] |= __ldg(pl + 32 * i);
+            }
+        }
+        if (eos_word >= 0 && eos_word < kObWords && (eos_word & 31) == lane && q != p.dead && p.accept[q]) {
+#pragma unroll
+            for (int i = 0; i < kObWords / 32; ++i)
+                if ((eos_word >> 5) == i) acc[i] |= 1u << (p.eos_id & 31);
+        }
+        uint32_t* mrow = p.mask + static_cast<size_t>(r) * p.G + w0 + lane;
+#pragma unroll
+        for (int i = 0; i < kObWords / 32; ++i)
+            if (w0 + lane + 32 * i < p.G) mrow[32 * i] = acc[i];
+        __syncwarp();  // the list is rewritten for the next row
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Survivors among the tokens of two or more bytes.
+template <typename TabT, bool FULL>
+__device__ __forceinline__ void bucket_tasks(const WalkParams& p, const TabT* __restrict__ tab,
+                                             uint32_t Cs, const int32_t* s_gstart, int* s_next) {
+    const uint32_t dead = p.dead;
+    auto lookup = [&](uint32_t s, uint32_t c) -> uint32_t {
+        if (FULL) return tab[s * Cs + c];
+        return __ldg(tab + static_cast<size_t>(s) * Cs + c);
+    };
+    const int lane = threadIdx.x & 31;
+    const int n_sorted = s_gstart[256];
+    const int nwin = (n_sorted + 31) >> 5;
+    const int nrows = p.q_end - p.q_begin;
+    const int parts = (nrows + kStatesPerTask - 1) / kStatesPerTask;
+    const int64_t ntasks = static_cast<int64_t>(nwin) * parts;
+    // Tasks cost very differently (a window of rare keys holds many keys, each with its own
+    // scan of the states).  Task i of this CTA is task i * gridDim.x + blockIdx.x, so that
+    // neighbouring windows go to different SMs; inside the CTA warps draw from a counter.
+    while (true) {
+        int i = 0;
+        if (lane == 0) i = atomicAdd(s_next, 1);
+        i = __shfl_sync(kFullWarp, i, 0);
+        const int64_t t = static_cast<int64_t>(i) * gridDim.x + blockIdx.x;
+        if (t >= ntasks) break;
+        const int win = static_cast<int>(t / parts);
+        const int part = static_cast<int>(t - static_cast<int64_t>(win) * parts);
+        const int pos = win * 32 + lane;
+        uint4 rec = make_uint4(0, 0, 0, 0);
+        int32_t id = -1;
+        if (pos < n_sorted) {
+            rec = __ldg(p.srec + pos);
+            id = __ldg(p.sid + pos);
+        }
+        const int len = rec.x & 0xFFu;
+        const bool active = id >= 0 && len >= 2;
+        uint32_t todo = __ballot_sync(kFullWarp, active);
+        if (todo == 0) continue;
+        // first-byte class: the last c with gstart[c] <= pos
+        int c0 = 0;
+#pragma unroll
+        for (int step = 128; step > 0; step >>= 1)
+            if (s_gstart[c0 + step] <= pos) c0 += step;
+        const uint32_t key = (static_cast<uint32_t>(c0) << 8) | ((rec.x >> 8) & 0xFFu);
+        const uint32_t bit = 1u << (id & 31);
+        const int word = id >> 5;
+        while (todo) {
+            const uint32_t kl = __shfl_sync(kFullWarp, key, __ffs(todo) - 1);
+            const bool same = active && key == kl;
+            todo &= ~__ballot_sync(kFullWarp, same);
+            const uint32_t c0l = kl >> 8, c1l = kl & 0xFFu;
+            for (int g = 0; g < kStatesPerTask / 32; ++g) {
+                const int rbase = part * kStatesPerTask + g * 32;
+                if (rbase >= nrows) break;
+                uint32_t s2 = dead;
+                if (rbase + lane < nrows) s2 = lookup(lookup(p.q_begin + rbase + lane, c0l), c1l);
+                uint32_t m = __ballot_sync(kFullWarp, s2 != dead);
+                while (m) {
+                    const int l = __ffs(m) - 1;
+                    m &= m - 1;
+                    const uint32_t s = __shfl_sync(kFullWarp, s2, l);
+                    bool go = same && len > 2;
+                    uint32_t st = walk_rest<TabT, FULL, 2>(tab, Cs, dead, rec, len, s, go);
+                    if (go)  // longer than the inline record and still alive
+                        st = raw_walk(p, st, p.vocab_offsets[id], p.vocab_offsets[id + 1], kInlineBytes);
+                    if (same && st != dead)
+                        atomicOr(p.mask + static_cast<size_t>(rbase + l) * p.G + word, bit);
+                }
+            }
+        }
+    }
+}
+
+template <typename TabT>
+__global__ void __launch_bounds__(kWalkThreads, 1) walk_buckets(const WalkParams p) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    __shared__ uint64_t bar;
+    __shared__ int32_t s_gstart[260];
+    __shared__ int s_next;
+    if (p.meta->any_bad != 0) return;  // mask_onebyte did the whole build
+    TabT* stab = reinterpret_cast<TabT*>(smem_raw);
+    const uint32_t Cs = p.meta->Cs;
+    for (int i = threadIdx.x; i < 257; i += kWalkThreads) s_gstart[i] = p.gstart[i];
+    if (threadIdx.x == 0) s_next = 0;
+    bool full;
+    if (!stage_table<TabT>(p, stab, &bar, p.smem_cap, Cs, full)) return;
+    __syncthreads();
+    if (full)
+        bucket_tasks<TabT, true>(p, stab, Cs, s_gstart, &s_next);
+    else
+        bucket_tasks<TabT, false>(p, static_cast<const TabT*>(p.table), Cs, s_gstart, &s_next);
+}
+
+// ---------------------------------------------------------------------------------------
+template <typename TabT>
+cudaError_t launch_bucket(const WalkParams& p, int sms, cudaStream_t stream) {
+    const int nrows = p.q_end - p.q_begin;
+    // mask_onebyte: 128 bitmask words per block column, rows spread over up to 16 block rows
+    const int ycap = (nrows + 7) / 8;
+    dim3 grid_a((p.G + kObWords - 1) / kObWords, ycap < 16 ? ycap : 16);
+    mask_onebyte<<<grid_a, kObThreads, 0, stream>>>(p);
+    auto k1 = walk_buckets<TabT>;
+    cudaError_t e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(p.smem_cap));
+    if (e != cudaSuccess) return e;
+    k1<<<sms, kWalkThreads, p.smem_cap, stream>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+}  // namespace fsm

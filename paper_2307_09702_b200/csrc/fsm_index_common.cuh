@@ -44,8 +44,11 @@ struct Workspace {
     int32_t* cursor2;    // [kKeys] placement cursors
     int32_t* start2;     // [kKeys] first sorted position of each (first class, second key)
     void* survivors;     // [kMaxSparseCtas][slices][256] survivor lists of the sparse walk
+    // bucket walk: bit planes of the one-byte tokens by class, live classes of every state
+    uint32_t* planes;    // [256][W] bit v of plane c: token v is the one byte of class c
+    uint32_t* live;      // [Q][8] bit c: state reads class c
     size_t bytes;        // everything above
-    size_t dense_bytes;  // without `survivors`: enough for the dense walk
+    size_t dense_bytes;  // the part in front of `survivors`: enough for the dense walk
 };
 
 inline size_t table_elem_bytes(int32_t Q) { return Q <= 65535 ? 2 : 4; }
@@ -83,6 +86,8 @@ inline Workspace carve(void* base, int32_t Q, int32_t N) {
     const size_t ctas = Q < kMaxSparseCtas ? Q : kMaxSparseCtas;
     const size_t slice_slots = (static_cast<size_t>(N) + 511) / 512 * 512;
     w.survivors = take(ctas * slice_slots * (Q <= 65535 ? 4 : 8));
+    w.planes = reinterpret_cast<uint32_t*>(take(256 * (G32 / 32) * sizeof(uint32_t)));
+    w.live = reinterpret_cast<uint32_t*>(take(static_cast<size_t>(Q) * 8 * sizeof(uint32_t)));
     w.bytes = off;
     return w;
 }
@@ -107,6 +112,9 @@ struct WalkParams {
     const int32_t* count2;
     const int32_t* start2;
     int32_t* row_ctr;
+    // bucket walk
+    const uint32_t* planes;
+    const uint32_t* live;
     // outputs
     uint32_t* mask;
     void* next;

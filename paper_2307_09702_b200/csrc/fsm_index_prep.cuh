@@ -100,10 +100,11 @@ __global__ void __launch_bounds__(256) derive_classes(const uint64_t* __restrict
 }
 
 // ---------------------------------------------------------------------------- 3
-// Blocks [0, row_blocks) compress and verify table rows; the remaining blocks write the
-// class records of the tokens in token order (dense walk; the launch for the sparse walk
-// has no such blocks).  Column C of the compressed table (the null class) and the padding
-// columns lead to the dead state, as does the whole row of the dead state.
+// Blocks [0, row_blocks) compress and verify table rows and, for the bucket walk, note
+// which classes each state reads (`live`); the remaining blocks write the class records of
+// the tokens in token order (dense walk; the launch for the other walks has no such
+// blocks).  Column C of the compressed table (the null class) and the padding columns lead
+// to the dead state, as does the whole row of the dead state.
 template <typename TabT>
 __global__ void __launch_bounds__(256)
 prepare_inputs(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab_bytes,
@@ -111,7 +112,7 @@ prepare_inputs(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vo
                int32_t N, int32_t dead, int32_t eos_id, int row_blocks, IndexMeta* meta,
                const uint8_t* __restrict__ cls, const uint8_t* __restrict__ class_rep,
                TabT* __restrict__ table, uint4* __restrict__ tok_cls,
-               uint8_t* __restrict__ tok_len, int32_t* status) {
+               uint8_t* __restrict__ tok_len, uint32_t* __restrict__ live, int32_t* status) {
     const int C = meta->C, Cs = meta->Cs;
     if (static_cast<int>(blockIdx.x) < row_blocks) {
         __shared__ int32_t row[256];
@@ -127,6 +128,12 @@ prepare_inputs(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vo
             for (int c = threadIdx.x; c < Cs; c += 256) {
                 int32_t v = (q == dead || c >= C) ? dead : row[s_rep[c]];
                 table[static_cast<size_t>(q) * Cs + c] = static_cast<TabT>(v);
+            }
+            if (live != nullptr) {  // thread c: does q read class c?
+                const int c = threadIdx.x;
+                const bool reads = q != dead && c < C && row[s_rep[c < C ? c : 0]] != dead;
+                const uint32_t m = __ballot_sync(kFullWarp, reads);
+                if ((c & 31) == 0) live[static_cast<size_t>(q) * 8 + (c >> 5)] = m;
             }
         }
         if (__syncthreads_or(bad) && threadIdx.x == 0) {
@@ -230,7 +237,7 @@ __global__ void __launch_bounds__(kSortThreads)
 count_keys(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vocab_offsets,
            int64_t vocab_nbytes, int32_t N, int32_t eos_id, const IndexMeta* __restrict__ meta,
            const uint8_t* __restrict__ cls, int32_t* __restrict__ gcount,
-           int32_t* __restrict__ count2, int32_t* status) {
+           int32_t* __restrict__ count2, uint32_t* __restrict__ planes, int32_t* status) {
     extern __shared__ int s_cnt[];  // [kKeys]
     __shared__ int hist[256];
     __shared__ uint8_t s_cls[256];
@@ -241,6 +248,16 @@ count_keys(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ 
     const bool two = meta->two_level != 0;
     const int nkeys = two ? kKeys : 256;
     for (int i = threadIdx.x; i < nkeys; i += kSortThreads) s_cnt[i] = 0;
+    // bucket walk: plane c holds the bits of the one-byte tokens of class c; the block owns
+    // 32 words of every plane and clears them first
+    const int W = (N + 31) / 32;
+    if (planes != nullptr) {
+        const int C = meta->C;
+        for (int i = threadIdx.x; i < C * 32; i += kSortThreads) {
+            const int word = blockIdx.x * 32 + (i & 31);
+            if (word < W) planes[static_cast<size_t>(i >> 5) * W + word] = 0;
+        }
+    }
     __syncthreads();
     bool bad = false;
     const int64_t v = static_cast<int64_t>(blockIdx.x) * kSortTokens + threadIdx.x;
@@ -248,6 +265,12 @@ count_keys(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ 
     if (t.len > 0) {
         atomicAdd(&hist[t.first], 1);
         atomicAdd(&s_cnt[bucket_key(two, t.first, t.second_key)], 1);
+    }
+    if (planes != nullptr) {
+        const bool one = t.len == 1;
+        const uint32_t peers = __match_any_sync(kFullWarp, one ? t.first : 0xFFFF);
+        if (one && (threadIdx.x & 31) == __ffs(peers) - 1)
+            planes[static_cast<size_t>(t.first) * W + (v >> 5)] = peers;
     }
     if (__syncthreads_or(bad) && threadIdx.x == 0) raise_flag(status, FSM_FLAG_OFFSETS);
     for (int i = threadIdx.x; i < nkeys; i += kSortThreads)

@@ -378,11 +378,11 @@ __device__ void raw_rows(const WalkParams& p) {
         OutT* nrow = HAS_OUT ? static_cast<OutT*>(p.next) + static_cast<size_t>(r) * p.N : nullptr;
         uint32_t* mrow = p.mask + static_cast<size_t>(r) * p.G;
         if (HAS_OUT)
-            for (int i = threadIdx.x; i < p.N; i += kWalkThreads) nrow[i] = static_cast<OutT>(dead);
-        for (int i = threadIdx.x; i < p.G; i += kWalkThreads) mrow[i] = 0;
+            for (int i = threadIdx.x; i < p.N; i += blockDim.x) nrow[i] = static_cast<OutT>(dead);
+        for (int i = threadIdx.x; i < p.G; i += blockDim.x) mrow[i] = 0;
         __syncthreads();  // orders the fill before the scattered stores
         if (q != p.dead) {
-            for (int v = threadIdx.x; v < p.N; v += kWalkThreads) {
+            for (int v = threadIdx.x; v < p.N; v += blockDim.x) {
                 if (v == p.eos_id) continue;
                 const int64_t o0 = p.vocab_offsets[v], o1 = p.vocab_offsets[v + 1];
                 if (o0 < 0 || o1 <= o0 || o1 > p.vocab_nbytes) continue;

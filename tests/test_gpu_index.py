@@ -15,9 +15,9 @@ if torch.cuda.is_available():
     from gpu_util import THREADS, check_index, gpu_index, mask_np, next_np
 
 
-@pytest.fixture(autouse=True, params=[1, 2], ids=["dense", "bucketed"])
+@pytest.fixture(autouse=True, params=[1, 2, 3], ids=["dense", "rowwise", "bucket"])
 def _walk_algorithm(request):
-    """Every case runs with both walk kernels; knobs are reset afterwards."""
+    """Every case runs with each walk algorithm; knobs are reset afterwards."""
     fg.fsm_debug_set(6, request.param)
     yield
     for key in (1, 2, 3, 4, 6):
