@@ -42,6 +42,20 @@ void profile_end(int slot, cudaStream_t stream);
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 #ifdef __CUDACC__
+// Plain launch on `stream` through the extensible launch API.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_on(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                      cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
+#ifdef __CUDACC__
 __device__ __forceinline__ void raise_flag(int32_t* status_word, int flag) {
     if (status_word != nullptr) atomicOr(status_word, flag);
 }

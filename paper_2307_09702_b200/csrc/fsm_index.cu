@@ -3,14 +3,14 @@
 //
 // Launches on the caller's stream, no host synchronisation:
 //   1. hash_columns    one pass over delta: a 64-bit hash of each of the 256 byte columns
-//   2. derive_classes  bytes with equal column hashes share a byte class
-//   3. prepare_inputs  class-compressed table [Q x Cs] with exact verification that every
-//                      byte's column equals its class representative's column; token
-//                      records (dense walk) or bucket counts (sparse walk)
-//   3b. count_keys, scan_keys, sort_tokens   sparse walk only: tokens sorted by (first,
-//                      second) byte class
+//   2. prepare_all     bytes with equal column hashes share a byte class; class-compressed
+//                      table [Q x Cs] with exact verification that every byte's column
+//                      equals its class representative's column; token records (dense
+//                      walk) or bucket key counts (work-avoiding walks)
+//   3. sort_all        work-avoiding walks only: tokens sorted by (first, second) byte class
 //   4. walk            dense: every (state, token) pair walked by warp tiles;
-//      walk_sparse     only tokens of readable buckets walked, rows pre-filled with dead
+//      walk_sparse     only tokens of readable buckets walked, rows assembled slice by slice;
+//      mask_onebyte + walk_buckets   bitmask-only builds
 // If verification in 3 fails (a 64-bit hash collision) the walk reads the uncompressed
 // table instead, so the result is exact in every case.
 #include "fsm_index_common.cuh"
@@ -76,40 +76,54 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
                         sparse_table_offset<int32_t>(N) + 4096 <= static_cast<size_t>(dev.smem_optin - 2048);
 
     const int hash_blocks = Q < kHashBlocks ? Q : kHashBlocks;
-    hash_columns<<<hash_blocks, 256 * kHashRowLanes, 0, stream>>>(
-        dfa_trans, Q, dead_state, ws.partial, tune.weak_hash, ws.gcount, ws.count2, ws.cursor2,
-        ws.row_ctr, status_word);
-    derive_classes<<<1, 256, 0, stream>>>(ws.partial, hash_blocks, ws.meta, ws.cls, ws.class_rep);
-    const int row_blocks = Q < 16 * dev.sm_count ? Q : 16 * dev.sm_count;
-    const int tok_blocks = sparse ? 0 : (G * 32 + 255) / 256;  // dense walk: token records
+    if (launch_on(hash_columns, dim3(hash_blocks), dim3(256 * kHashRowLanes), 0, stream,
+                          dfa_trans, Q, dead_state, ws.partial, tune.weak_hash, ws.meta, ws.gcount,
+                          ws.count2, ws.cursor2, ws.row_ctr, status_word) != cudaSuccess)
+        return FSM_ERR_CUDA;
+    // prepare_all: blocks share the table rows and the tokens
+    const int nchunks = (N + kPrepTokens - 1) / kPrepTokens;
+    const int row_passes = (Q + kPrepRows - 1) / kPrepRows;
+    int prep_blocks = row_passes > nchunks ? row_passes : nchunks;
+    if (prep_blocks > dev.sm_count) prep_blocks = dev.sm_count;
+    uint4* tok_cls = sparse ? nullptr : ws.tok_cls;  // dense walk: token records
+    int32_t* count2 = sparse ? ws.count2 : nullptr;  // work-avoiding walks: bucket keys
     uint32_t* live = bucket ? ws.live : nullptr;
     uint32_t* planes = bucket ? ws.planes : nullptr;
-    if (wide)
-        prepare_inputs<int32_t><<<row_blocks + tok_blocks, 256, 0, stream>>>(
-            dfa_trans, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
-            row_blocks, ws.meta, ws.cls, ws.class_rep, static_cast<int32_t*>(ws.table),
-            ws.tok_cls, ws.tok_len, live, status_word);
-    else
-        prepare_inputs<uint16_t><<<row_blocks + tok_blocks, 256, 0, stream>>>(
-            dfa_trans, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
-            row_blocks, ws.meta, ws.cls, ws.class_rep, static_cast<uint16_t*>(ws.table),
-            ws.tok_cls, ws.tok_len, live, status_word);
-    if (sparse) {
-        const int sort_blocks = (N + kSortTokens - 1) / kSortTokens;
-        const size_t key_smem = kKeys * sizeof(int);
-        if (cudaFuncSetAttribute(count_keys, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(key_smem)) != cudaSuccess ||
-            cudaFuncSetAttribute(sort_tokens, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(key_smem)) != cudaSuccess)
+    const size_t key_smem = sparse ? kKeys * sizeof(int) : 0;
+    const size_t sort_smem = (kKeysPad + kKeys) * sizeof(int);
+    if (wide) {
+        auto k = prepare_all<int32_t>;
+        if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kKeys * sizeof(int))) != cudaSuccess)
             return FSM_ERR_CUDA;
-        count_keys<<<sort_blocks, kSortThreads, key_smem, stream>>>(
-            vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, ws.meta, ws.cls, ws.gcount,
-            ws.count2, planes, status_word);
-        scan_keys<<<kTwoLevelMaxC + 1, 256, 0, stream>>>(ws.meta, ws.gcount, ws.count2, ws.gstart,
-                                                         ws.start2);
-        sort_tokens<<<sort_blocks, kSortThreads, key_smem, stream>>>(
-            vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, ws.meta, ws.cls, ws.start2,
-            ws.cursor2, ws.srec, ws.sid);
+        if (launch_on(k, dim3(prep_blocks), dim3(kPrepThreads), key_smem, stream, dfa_trans,
+                              vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
+                              ws.partial, hash_blocks, ws.meta, ws.cls, static_cast<int32_t*>(ws.table),
+                              tok_cls, ws.tok_len, live, ws.gcount, count2, planes,
+                              status_word) != cudaSuccess)
+            return FSM_ERR_CUDA;
+    } else {
+        auto k = prepare_all<uint16_t>;
+        if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kKeys * sizeof(int))) != cudaSuccess)
+            return FSM_ERR_CUDA;
+        if (launch_on(k, dim3(prep_blocks), dim3(kPrepThreads), key_smem, stream, dfa_trans,
+                              vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
+                              ws.partial, hash_blocks, ws.meta, ws.cls, static_cast<uint16_t*>(ws.table),
+                              tok_cls, ws.tok_len, live, ws.gcount, count2, planes,
+                              status_word) != cudaSuccess)
+            return FSM_ERR_CUDA;
+    }
+    if (sparse) {
+        if (cudaFuncSetAttribute(sort_all, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(sort_smem)) != cudaSuccess)
+            return FSM_ERR_CUDA;
+        const int sort_blocks = nchunks < dev.sm_count ? nchunks : dev.sm_count;
+        if (launch_on(sort_all, dim3(sort_blocks), dim3(kPrepThreads), sort_smem, stream,
+                              vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, ws.meta, ws.cls,
+                              ws.count2, ws.cursor2, ws.start2, ws.gstart, ws.srec,
+                              ws.sid) != cudaSuccess)
+            return FSM_ERR_CUDA;
     }
     if (cudaGetLastError() != cudaSuccess) return FSM_ERR_CUDA;
 

@@ -222,13 +222,13 @@ cudaError_t launch_bucket(const WalkParams& p, int sms, cudaStream_t stream) {
     // mask_onebyte: 128 bitmask words per block column, rows spread over up to 16 block rows
     const int ycap = (nrows + 7) / 8;
     dim3 grid_a((p.G + kObWords - 1) / kObWords, ycap < 16 ? ycap : 16);
-    mask_onebyte<<<grid_a, kObThreads, 0, stream>>>(p);
-    auto k1 = walk_buckets<TabT>;
-    cudaError_t e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(p.smem_cap));
+    cudaError_t e = launch_on(mask_onebyte, grid_a, dim3(kObThreads), 0, stream, p);
     if (e != cudaSuccess) return e;
-    k1<<<sms, kWalkThreads, p.smem_cap, stream>>>(p);
-    return cudaGetLastError();
+    auto k1 = walk_buckets<TabT>;
+    e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(p.smem_cap));
+    if (e != cudaSuccess) return e;
+    return launch_on(k1, dim3(sms), dim3(kWalkThreads), p.smem_cap, stream, p);
 }
 
 }  // namespace

@@ -6,7 +6,7 @@
 namespace fsm {
 namespace {
 
-constexpr int kHashBlocks = 64;
+constexpr int kHashBlocks = 32;
 constexpr int kMaxCs = 264;             // 256 classes + the null class, rounded up to 8
 constexpr int kWalkThreads = 1024;
 constexpr int kWalkWarps = kWalkThreads / 32;
@@ -28,7 +28,6 @@ struct IndexMeta {
 struct Workspace {
     IndexMeta* meta;
     uint8_t* cls;        // [256] byte -> class
-    uint8_t* class_rep;  // [256] class -> representative byte
     uint64_t* partial;   // [kHashBlocks][256] column hash partial sums
     void* table;         // [Q][Cs] of TabT
     // dense walk: token records in token order (aliases the sparse walk's arrays)
@@ -65,7 +64,6 @@ inline Workspace carve(void* base, int32_t Q, int32_t N) {
     const size_t G32 = (static_cast<size_t>(N) + 31) / 32 * 32;
     w.meta = reinterpret_cast<IndexMeta*>(take(sizeof(IndexMeta)));
     w.cls = take(256);
-    w.class_rep = take(256);
     w.partial = reinterpret_cast<uint64_t*>(take(sizeof(uint64_t) * kHashBlocks * 256));
     w.table = take(static_cast<size_t>(Q) * kMaxCs * table_elem_bytes(Q));
     const size_t dense_bytes = G32 * sizeof(uint4) + G32;
@@ -138,19 +136,26 @@ __device__ __forceinline__ int bucket_key(bool two_level, int first, int second_
     return two_level ? first * kKeyStride + second_key : first;
 }
 
-// Bounds-checked view of one token for the token-side preparation kernels.
+// Bounds-checked view of one token for the token-side preparation kernels.  The raw part
+// (offsets and first bytes) does not depend on the byte classes, so it can be fetched
+// before they are known.
+struct TokenRaw {
+    int64_t start;
+    int len;          // min(length, kInlineBytes + 1); 0 = not bucketed (empty, EOS, bad offsets)
+    uint32_t b0, b1;  // first two bytes
+};
 struct TokenInfo {
     int64_t start;
-    int len;         // min(length, kInlineBytes + 1); 0 = not bucketed (empty, EOS, bad offsets)
+    int len;
     int first;       // class of byte 0
     int second_key;  // 0 for one-byte tokens, else 1 + class of byte 1
 };
 
-__device__ __forceinline__ TokenInfo token_info(const uint8_t* __restrict__ vocab_bytes,
-                                                const int32_t* __restrict__ vocab_offsets,
-                                                int64_t vocab_nbytes, int32_t N, int32_t eos_id,
-                                                const uint8_t* s_cls, int64_t v, bool* bad) {
-    TokenInfo t = {0, 0, 0, 0};
+__device__ __forceinline__ TokenRaw token_raw(const uint8_t* __restrict__ vocab_bytes,
+                                              const int32_t* __restrict__ vocab_offsets,
+                                              int64_t vocab_nbytes, int32_t N, int32_t eos_id,
+                                              int64_t v, bool* bad) {
+    TokenRaw t = {0, 0, 0, 0};
     if (v < N && v != eos_id) {
         const int64_t o0 = vocab_offsets[v], o1 = vocab_offsets[v + 1];
         if (o0 < 0 || o1 < o0 || o1 > vocab_nbytes) {
@@ -158,10 +163,17 @@ __device__ __forceinline__ TokenInfo token_info(const uint8_t* __restrict__ voca
         } else if (o1 > o0) {
             t.start = o0;
             t.len = static_cast<int>(min(o1 - o0, static_cast<int64_t>(kInlineBytes + 1)));
-            t.first = s_cls[vocab_bytes[o0]];
-            if (t.len > 1) t.second_key = 1 + s_cls[vocab_bytes[o0 + 1]];
+            t.b0 = vocab_bytes[o0];
+            if (t.len > 1) t.b1 = vocab_bytes[o0 + 1];
         }
     }
+    return t;
+}
+
+__device__ __forceinline__ TokenInfo token_classify(const TokenRaw& r, const uint8_t* s_cls) {
+    TokenInfo t = {r.start, r.len, 0, 0};
+    if (r.len > 0) t.first = s_cls[r.b0];
+    if (r.len > 1) t.second_key = 1 + s_cls[r.b1];
     return t;
 }
 

@@ -154,8 +154,7 @@ cudaError_t launch_walk(const WalkParams& p, int grid, cudaStream_t stream) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(p.smem_cap));
     if (e != cudaSuccess) return e;
-    kernel<<<grid, kWalkThreads, p.smem_cap, stream>>>(p);
-    return cudaGetLastError();
+    return launch_on(kernel, dim3(grid), dim3(kWalkThreads), p.smem_cap, stream, p);
 }
 
 template <typename TabT>

@@ -1,4 +1,10 @@
 // Preparation kernels of the index build: byte classes, compressed table, token layouts.
+//
+// Three launches: hash_columns (a hash of each byte column of delta), prepare_all (every
+// block derives the byte classes from the hashes, then the blocks share the table rows and
+// the tokens) and, for the work-avoiding walks, sort_all (every block scans the key counts,
+// then the blocks share the tokens).  The small serial steps are repeated by every block
+// instead of being launches of their own.
 #pragma once
 
 #include "fsm_index_common.cuh"
@@ -10,29 +16,33 @@ namespace {
 // Thread (b, lane) owns byte column b of delta for rows lane, lane+4, ... of the block's
 // share (coalesced 1 KB row reads).  The per-column hash is a wrap-around sum of mixed
 // (row, value) pairs, so equal columns hash alike and partial sums simply add.  The
-// blocks also clear the counters of the token sort.
+// blocks also clear the counters of the token sort and the flag of the class check.
 constexpr int kHashRowLanes = 4;
 
 __global__ void __launch_bounds__(256 * kHashRowLanes)
 hash_columns(const int32_t* __restrict__ trans, int32_t Q, int32_t dead,
-             uint64_t* __restrict__ partial, int weak, int32_t* __restrict__ gcount,
-             int32_t* __restrict__ count2, int32_t* __restrict__ cursor2,
-             int32_t* __restrict__ row_ctr, int32_t* status) {
-    if (blockIdx.x == 0 && threadIdx.x == 0) *row_ctr = 0;
+             uint64_t* __restrict__ partial, int weak, IndexMeta* meta,
+             int32_t* __restrict__ gcount, int32_t* __restrict__ count2,
+             int32_t* __restrict__ cursor2, int32_t* __restrict__ row_ctr, int32_t* status) {
     __shared__ uint64_t part[kHashRowLanes][256];
     const int b = threadIdx.x & 255, rl = threadIdx.x >> 8;
+    uint64_t h = 0;
+    bool bad = false;
+#pragma unroll 4
+    for (int q = blockIdx.x * kHashRowLanes + rl; q < Q; q += gridDim.x * kHashRowLanes) {
+        const int32_t v = trans[static_cast<size_t>(q) * 256 + b];
+        if (q == dead) continue;
+        bad |= static_cast<uint32_t>(v) >= static_cast<uint32_t>(Q);
+        h += mix64((static_cast<uint64_t>(q) << 32) | static_cast<uint32_t>(v));
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        *row_ctr = 0;
+        meta->any_bad = 0;
+    }
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < kKeys; i += gridDim.x * blockDim.x) {
         count2[i] = 0;
         cursor2[i] = 0;
         if (i < 256) gcount[i] = 0;
-    }
-    uint64_t h = 0;
-    bool bad = false;
-    for (int q = blockIdx.x * kHashRowLanes + rl; q < Q; q += gridDim.x * kHashRowLanes) {
-        if (q == dead) continue;
-        int32_t v = trans[static_cast<size_t>(q) * 256 + b];
-        bad |= static_cast<uint32_t>(v) >= static_cast<uint32_t>(Q);
-        h += mix64((static_cast<uint64_t>(q) << 32) | static_cast<uint32_t>(v));
     }
     part[rl][b] = h;
     const int any_bad = __syncthreads_or(bad);
@@ -46,276 +56,351 @@ hash_columns(const int32_t* __restrict__ trans, int32_t Q, int32_t dead,
 }
 
 // ---------------------------------------------------------------------------- 2
-// One block.  Bytes whose column hashes are equal form a class, represented by the
-// smallest such byte; class ids are the ranks of the representatives.  Equal hashes
-// are found through a small open-addressing table in shared memory.
-__global__ void __launch_bounds__(256) derive_classes(const uint64_t* __restrict__ partial,
-                                                     int nblocks, IndexMeta* meta, uint8_t* cls,
-                                                     uint8_t* class_rep) {
+constexpr int kPrepThreads = 1024;
+constexpr int kPrepRows = kPrepThreads / 256;  // table rows handled per pass
+constexpr int kPrepTokens = kPrepThreads;      // tokens handled per pass
+
+// Byte classes from the column hashes, computed by the first 256 threads of a block
+// (thread = byte) into shared memory.  Bytes whose hashes are equal form a class,
+// represented by the smallest such byte; class ids are the ranks of the representatives.
+// Equal hashes are found through a small open-addressing table.  Returns the number of
+// classes; ends with a barrier.
+struct ClassScratch {
+    unsigned long long keys[1024];
+    int min_byte[1024];
+    uint32_t rep_bits[8];
+};
+
+__device__ __forceinline__ int derive_classes(const uint64_t* __restrict__ partial, int nparts,
+                                              ClassScratch& cs, uint8_t* s_cls, uint8_t* s_rep) {
     constexpr int kSlots = 1024;
-    __shared__ unsigned long long keys[kSlots];
-    __shared__ int min_byte[kSlots];
-    __shared__ uint32_t rep_bits[8];
     constexpr unsigned long long kEmpty = ~0ull;
     const int b = threadIdx.x;
-    uint64_t sum = 0;
+    for (int i = b; i < kSlots; i += blockDim.x) {
+        cs.keys[i] = kEmpty;
+        cs.min_byte[i] = 256;
+    }
+    __syncthreads();
+    int slot = 0;
+    if (b < 256) {
+        uint64_t sum = 0;
 #pragma unroll 8
-    for (int k = 0; k < nblocks; ++k) sum += partial[k * 256 + b];
-    // kEmpty marks a free slot; folding that one value onto its neighbour can only merge
-    // two classes, which the exact verification of the next kernel would catch.
-    const unsigned long long key = (sum == kEmpty) ? sum - 1 : sum;
-    for (int i = b; i < kSlots; i += 256) {
-        keys[i] = kEmpty;
-        min_byte[i] = 256;
+        for (int k = 0; k < nparts; ++k) sum += partial[k * 256 + b];
+        // kEmpty marks a free slot; folding that one value onto its neighbour can only
+        // merge two classes, which the exact verification of the table rows would catch.
+        const unsigned long long key = (sum == kEmpty) ? sum - 1 : sum;
+        // at most 256 distinct keys in 1024 slots: linear probing ends within kSlots steps
+        slot = static_cast<int>((key ^ (key >> 29)) & (kSlots - 1));
+        for (int probe = 0; probe < kSlots; ++probe) {
+            const unsigned long long was = atomicCAS(&cs.keys[slot], kEmpty, key);
+            if (was == kEmpty || was == key) break;
+            slot = (slot + 1) & (kSlots - 1);
+        }
+        atomicMin(&cs.min_byte[slot], b);
     }
     __syncthreads();
-    // at most 256 distinct keys in 1024 slots: linear probing ends within kSlots steps
-    int slot = static_cast<int>((key ^ (key >> 29)) & (kSlots - 1));
-    for (int probe = 0; probe < kSlots; ++probe) {
-        const unsigned long long was = atomicCAS(&keys[slot], kEmpty, key);
-        if (was == kEmpty || was == key) break;
-        slot = (slot + 1) & (kSlots - 1);
+    int r = 0;
+    if (b < 256) {  // warps 0..7, whole warps
+        r = cs.min_byte[slot];
+        const uint32_t m = __ballot_sync(kFullWarp, r == b);
+        if ((b & 31) == 0) cs.rep_bits[b >> 5] = m;
     }
-    atomicMin(&min_byte[slot], b);
     __syncthreads();
-    const int r = min_byte[slot];
-    const bool is_rep = (r == b);
-    const uint32_t m = __ballot_sync(kFullWarp, is_rep);
-    if ((b & 31) == 0) rep_bits[b >> 5] = m;
+    int C = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) C += __popc(cs.rep_bits[w]);
+    if (b < 256) {
+        int id = __popc(cs.rep_bits[r >> 5] & ((1u << (r & 31)) - 1u));
+        for (int w = 0; w < (r >> 5); ++w) id += __popc(cs.rep_bits[w]);
+        s_cls[b] = static_cast<uint8_t>(id);
+        if (r == b) s_rep[id] = static_cast<uint8_t>(b);
+    }
     __syncthreads();
-    int id = __popc(rep_bits[r >> 5] & ((1u << (r & 31)) - 1u));
-    for (int w = 0; w < (r >> 5); ++w) id += __popc(rep_bits[w]);
-    cls[b] = static_cast<uint8_t>(id);
-    if (is_rep) class_rep[id] = static_cast<uint8_t>(b);
-    if (b == 0) {
-        int C = 0;
-        for (int w = 0; w < 8; ++w) C += __popc(rep_bits[w]);
-        meta->C = C;
-        meta->Cs = (C + 1 + 7) & ~7;
-        // 256 distinct columns leave no byte value for the null class: such a table
-        // is walked uncompressed.
-        meta->any_bad = (C > 255) ? 1 : 0;
-        meta->two_level = (C <= kTwoLevelMaxC) ? 1 : 0;
+    return C;
+}
+
+// Every block derives the classes; block 0 publishes them.  Then the blocks share
+//   - the table rows: compressed row [Cs] with exact verification that every byte's column
+//     equals its class representative's column, and (bucket walk) the classes the state
+//     reads.  Column C (the null class) and the padding columns lead to the dead state, as
+//     does the whole row of the dead state;
+//   - the tokens: class records in token order (dense walk), or the counts of the bucket
+//     keys (work-avoiding walks: class of the first byte and, with at most kTwoLevelMaxC
+//     classes, class of the second byte; key 0 = one-byte token) and (bucket walk) the bit
+//     planes of the one-byte tokens.  Keys are counted in shared memory over all tokens
+//     of the block, so that global memory sees one atomic per block and key: tokens that
+//     start with a space are a third of a BPE vocabulary and would otherwise all hit the
+//     same few counters.
+template <typename TabT>
+__global__ void __launch_bounds__(kPrepThreads)
+prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab_bytes,
+            const int32_t* __restrict__ vocab_offsets, int64_t vocab_nbytes, int32_t Q, int32_t N,
+            int32_t dead, int32_t eos_id, const uint64_t* __restrict__ partial, int nparts,
+            IndexMeta* meta, uint8_t* __restrict__ cls_out, TabT* __restrict__ table,
+            uint4* __restrict__ tok_cls, uint8_t* __restrict__ tok_len,
+            uint32_t* __restrict__ live, int32_t* __restrict__ gcount,
+            int32_t* __restrict__ count2, uint32_t* __restrict__ planes, int32_t* status) {
+    extern __shared__ int s_cnt[];  // [kKeys] when keys are counted
+    __shared__ ClassScratch cs;
+    __shared__ uint8_t s_cls[256], s_rep[256];
+    __shared__ int32_t rows[kPrepRows][256];
+    __shared__ int hist[256];
+    const int tid = threadIdx.x;
+    // What does not depend on the classes is fetched first: the block's first pass of table
+    // rows and of tokens.
+    int32_t row_first = dead;
+    if (static_cast<int>(blockIdx.x) * kPrepRows + (tid >> 8) < Q)
+        row_first = trans[(static_cast<size_t>(blockIdx.x) * kPrepRows + (tid >> 8)) * 256 + (tid & 255)];
+    bool bad_tok = false;
+    TokenRaw raw_first = {0, 0, 0, 0};
+    if (count2 != nullptr)
+        raw_first = token_raw(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id,
+                              static_cast<int64_t>(blockIdx.x) * kPrepTokens + tid, &bad_tok);
+    const int C = derive_classes(partial, nparts, cs, s_cls, s_rep);
+    const int Cs = (C + 1 + 7) & ~7;
+    const bool two = C <= kTwoLevelMaxC;
+    if (blockIdx.x == 0) {
+        if (tid < 256) cls_out[tid] = s_cls[tid];
+        if (tid == 0) {
+            meta->C = C;
+            meta->Cs = Cs;
+            meta->two_level = two ? 1 : 0;
+            // 256 distinct columns leave no byte value for the null class: such a table
+            // is walked uncompressed.
+            if (C > 255) atomicExch(&meta->any_bad, 1);
+        }
+    }
+    // ---- table rows, kPrepRows at a time (thread = (row lane, byte))
+    {
+        const int rl = tid >> 8, b = tid & 255;
+        bool bad = false;
+        for (int q0 = blockIdx.x * kPrepRows; q0 < Q; q0 += gridDim.x * kPrepRows) {
+            const int q = q0 + rl;
+            __syncthreads();
+            if (q < Q) {
+                const int32_t v = q0 == static_cast<int>(blockIdx.x) * kPrepRows
+                                      ? row_first
+                                      : trans[static_cast<size_t>(q) * 256 + b];
+                rows[rl][b] = clamp_state(v, Q, dead);
+            }
+            __syncthreads();
+            if (q < Q) {
+                if (q != dead) bad |= rows[rl][b] != rows[rl][s_rep[s_cls[b]]];
+                for (int c = b; c < Cs; c += 256) {
+                    const int32_t v = (q == dead || c >= C) ? dead : rows[rl][s_rep[c]];
+                    table[static_cast<size_t>(q) * Cs + c] = static_cast<TabT>(v);
+                }
+            }
+            if (live != nullptr) {  // thread (rl, c): does q read class c?
+                const bool reads = q < Q && q != dead && b < C && rows[rl][s_rep[b < C ? b : 0]] != dead;
+                const uint32_t m = __ballot_sync(kFullWarp, reads);
+                if ((b & 31) == 0 && q < Q) live[static_cast<size_t>(q) * 8 + (b >> 5)] = m;
+            }
+        }
+        if (__syncthreads_or(bad) && tid == 0) {
+            atomicExch(&meta->any_bad, 1);
+            raise_flag(status, FSM_FLAG_CLASS_SPLIT);
+        }
+    }
+    // ---- tokens in token order: class records of the dense walk
+    if (tok_cls != nullptr) {
+        const int64_t slots = (static_cast<int64_t>(N) + 31) / 32 * 32;
+        for (int64_t v = static_cast<int64_t>(blockIdx.x) * kPrepTokens + tid; v < slots;
+             v += static_cast<int64_t>(gridDim.x) * kPrepTokens) {
+            uint32_t w[4] = {static_cast<uint32_t>(C), 0, 0, 0};  // an empty token reads the null class
+            int len = 0;
+            if (v < N && v != eos_id) {
+                const int64_t o0 = vocab_offsets[v], o1 = vocab_offsets[v + 1];
+                if (o0 < 0 || o1 < o0 || o1 > vocab_nbytes) {
+                    raise_flag(status, FSM_FLAG_OFFSETS);
+                } else {
+                    len = static_cast<int>(min(o1 - o0, static_cast<int64_t>(kInlineBytes + 1)));
+                    const int n = min(len, kInlineBytes);
+                    if (n > 0) w[0] = 0;
+                    uint8_t raw[kInlineBytes];
+#pragma unroll
+                    for (int i = 0; i < kInlineBytes; ++i)  // independent loads, issued together
+                        raw[i] = i < n ? vocab_bytes[o0 + i] : 0;
+#pragma unroll
+                    for (int i = 0; i < kInlineBytes; ++i)
+                        if (i < n) w[i >> 2] |= static_cast<uint32_t>(s_cls[raw[i]]) << ((i & 3) * 8);
+                }
+            }
+            tok_cls[v] = make_uint4(w[0], w[1], w[2], w[3]);
+            tok_len[v] = static_cast<uint8_t>(len);
+        }
+    }
+    // ---- bucket keys of the tokens, kPrepTokens at a time
+    const int nchunks = (N + kPrepTokens - 1) / kPrepTokens;
+    if (count2 != nullptr && static_cast<int>(blockIdx.x) < nchunks) {
+        const int nkeys = two ? kKeys : 256;
+        const int W = (N + 31) / 32;
+        for (int i = tid; i < nkeys; i += kPrepThreads) s_cnt[i] = 0;
+        if (tid < 256) hist[tid] = 0;
+        bool bad = bad_tok;
+        for (int chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
+            // bucket walk: plane c holds the bits of the one-byte tokens of class c; the
+            // 32 words of this pass are cleared first
+            if (planes != nullptr)
+                for (int i = tid; i < C * 32; i += kPrepThreads) {
+                    const int word = chunk * 32 + (i & 31);
+                    if (word < W) planes[static_cast<size_t>(i >> 5) * W + word] = 0;
+                }
+            __syncthreads();
+            const int64_t v = static_cast<int64_t>(chunk) * kPrepTokens + tid;
+            const TokenRaw raw = chunk == static_cast<int>(blockIdx.x)
+                                     ? raw_first
+                                     : token_raw(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, v, &bad);
+            const TokenInfo t = token_classify(raw, s_cls);
+            if (t.len > 0) {
+                atomicAdd(&hist[t.first], 1);
+                atomicAdd(&s_cnt[bucket_key(two, t.first, t.second_key)], 1);
+            }
+            if (planes != nullptr) {
+                const bool one = t.len == 1;
+                const uint32_t peers = __match_any_sync(kFullWarp, one ? t.first : 0xFFFF);
+                if (one && (tid & 31) == __ffs(peers) - 1)
+                    planes[static_cast<size_t>(t.first) * W + (v >> 5)] = peers;
+            }
+        }
+        if (__syncthreads_or(bad) && tid == 0) raise_flag(status, FSM_FLAG_OFFSETS);
+        for (int i = tid; i < nkeys; i += kPrepThreads)
+            if (s_cnt[i] > 0) atomicAdd(&count2[i], s_cnt[i]);
+        if (tid < 256 && hist[tid] > 0) atomicAdd(&gcount[tid], hist[tid]);
     }
 }
 
 // ---------------------------------------------------------------------------- 3
-// Blocks [0, row_blocks) compress and verify table rows and, for the bucket walk, note
-// which classes each state reads (`live`); the remaining blocks write the class records of
-// the tokens in token order (dense walk; the launch for the other walks has no such
-// blocks).  Column C of the compressed table (the null class) and the padding columns lead
-// to the dead state, as does the whole row of the dead state.
-template <typename TabT>
-__global__ void __launch_bounds__(256)
-prepare_inputs(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab_bytes,
-               const int32_t* __restrict__ vocab_offsets, int64_t vocab_nbytes, int32_t Q,
-               int32_t N, int32_t dead, int32_t eos_id, int row_blocks, IndexMeta* meta,
-               const uint8_t* __restrict__ cls, const uint8_t* __restrict__ class_rep,
-               TabT* __restrict__ table, uint4* __restrict__ tok_cls,
-               uint8_t* __restrict__ tok_len, uint32_t* __restrict__ live, int32_t* status) {
-    const int C = meta->C, Cs = meta->Cs;
-    if (static_cast<int>(blockIdx.x) < row_blocks) {
-        __shared__ int32_t row[256];
-        __shared__ uint8_t s_cls[256], s_rep[256];
-        s_cls[threadIdx.x] = cls[threadIdx.x];
-        s_rep[threadIdx.x] = class_rep[threadIdx.x];
-        bool bad = false;
-        for (int q = blockIdx.x; q < Q; q += row_blocks) {
-            __syncthreads();
-            row[threadIdx.x] = clamp_state(trans[static_cast<size_t>(q) * 256 + threadIdx.x], Q, dead);
-            __syncthreads();
-            if (q != dead) bad |= row[threadIdx.x] != row[s_rep[s_cls[threadIdx.x]]];
-            for (int c = threadIdx.x; c < Cs; c += 256) {
-                int32_t v = (q == dead || c >= C) ? dead : row[s_rep[c]];
-                table[static_cast<size_t>(q) * Cs + c] = static_cast<TabT>(v);
-            }
-            if (live != nullptr) {  // thread c: does q read class c?
-                const int c = threadIdx.x;
-                const bool reads = q != dead && c < C && row[s_rep[c < C ? c : 0]] != dead;
-                const uint32_t m = __ballot_sync(kFullWarp, reads);
-                if ((c & 31) == 0) live[static_cast<size_t>(q) * 8 + (c >> 5)] = m;
-            }
-        }
-        if (__syncthreads_or(bad) && threadIdx.x == 0) {
-            atomicExch(&meta->any_bad, 1);
-            raise_flag(status, FSM_FLAG_CLASS_SPLIT);
-        }
-    } else {
-        const int64_t slots = (static_cast<int64_t>(N) + 31) / 32 * 32;
-        const int64_t v = static_cast<int64_t>(blockIdx.x - row_blocks) * 256 + threadIdx.x;
-        if (v >= slots) return;
-        uint32_t w[4] = {static_cast<uint32_t>(C), 0, 0, 0};  // an empty token reads the null class
-        int len = 0;
-        if (v < N && v != eos_id) {
-            const int64_t o0 = vocab_offsets[v], o1 = vocab_offsets[v + 1];
-            if (o0 < 0 || o1 < o0 || o1 > vocab_nbytes) {
-                raise_flag(status, FSM_FLAG_OFFSETS);
-            } else {
-                len = static_cast<int>(min(o1 - o0, static_cast<int64_t>(kInlineBytes + 1)));
-                const int n = min(len, kInlineBytes);
-                if (n > 0) w[0] = 0;
-                uint8_t raw[kInlineBytes];
-#pragma unroll
-                for (int i = 0; i < kInlineBytes; ++i)  // independent loads, issued together
-                    raw[i] = i < n ? vocab_bytes[o0 + i] : 0;
-#pragma unroll
-                for (int i = 0; i < kInlineBytes; ++i)
-                    if (i < n) w[i >> 2] |= static_cast<uint32_t>(cls[raw[i]]) << ((i & 3) * 8);
-            }
-        }
-        tok_cls[v] = make_uint4(w[0], w[1], w[2], w[3]);
-        tok_len[v] = static_cast<uint8_t>(len);
-    }
-}
+// Token order of the work-avoiding walks: a counting sort by bucket key.  Keys are
+// numbered first class major, so the exclusive prefix sum of the key counts is the first
+// sorted position of every key; every block computes it in shared memory (block 0
+// publishes it, and the first position of every first class, for the walk).  Then the
+// blocks share the tokens, kPrepTokens at a time: rank within the pass by shared-memory
+// counters, one global atomic per key present in the pass to reserve its positions.  A
+// record keeps the length and the classes of bytes 1..15; `sid` holds the token id.
+constexpr int kScanPer = (kKeys + kPrepThreads - 1) / kPrepThreads;  // keys per thread
+constexpr int kKeysPad = kScanPer * kPrepThreads;
 
-// ---------------------------------------------------------------------------- 3b
-// Token order of the sparse walk: a counting sort by bucket key - the class of the
-// first byte and, when there are at most kTwoLevelMaxC classes, the class of the second
-// byte (key 0 = one-byte token).  scan_keys turns the counts into first positions
-// (block c0 handles the keys of first class c0); count_keys / sort_tokens handle 1,024
-// tokens per block.  A record keeps the length and the classes of bytes 1..15; `sid` holds the
-// token id.
-__global__ void __launch_bounds__(256)
-scan_keys(const IndexMeta* __restrict__ meta, const int32_t* __restrict__ gcount,
-          const int32_t* __restrict__ count2, int32_t* __restrict__ gstart,
-          int32_t* __restrict__ start2) {
-    __shared__ int gst[257];
-    __shared__ int wsum[8];
-    if (threadIdx.x < 32) {  // exclusive prefix over the 256 class counts, 8 per lane
-        int local[8], sum = 0;
+__global__ void __launch_bounds__(kPrepThreads)
+sort_all(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vocab_offsets,
+         int64_t vocab_nbytes, int32_t N, int32_t eos_id, const IndexMeta* __restrict__ meta,
+         const uint8_t* __restrict__ cls, const int32_t* __restrict__ count2,
+         int32_t* __restrict__ cursor2, int32_t* __restrict__ start2,
+         int32_t* __restrict__ gstart, uint4* __restrict__ srec, int32_t* __restrict__ sid) {
+    extern __shared__ int s_sort[];  // s_start[kKeysPad], s_cnt[kKeys]
+    int* s_start = s_sort;
+    int* s_cnt = s_sort + kKeysPad;
+    __shared__ int wsum[kPrepThreads / 32];
+    __shared__ uint8_t s_cls[256];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // the block's first pass of tokens does not depend on the scan: fetch its bytes first
+    bool bad_first = false;
+    const TokenRaw raw_first = token_raw(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id,
+                                         static_cast<int64_t>(blockIdx.x) * kPrepTokens + tid, &bad_first);
+    uint8_t bytes_first[kInlineBytes];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            local[i] = sum;
-            sum += gcount[threadIdx.x * 8 + i];
-        }
-        int incl = sum;
+    for (int i = 2; i < kInlineBytes; ++i)
+        bytes_first[i] = i < raw_first.len ? vocab_bytes[raw_first.start + i] : 0;
+    bytes_first[0] = static_cast<uint8_t>(raw_first.b0);
+    bytes_first[1] = static_cast<uint8_t>(raw_first.b1);
+    if (tid < 256) s_cls[tid] = cls[tid];
+    const bool two = meta->two_level != 0;
+    const int nkeys = two ? kKeys : 256;
 #pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const int o = __shfl_up_sync(kFullWarp, incl, off);
-            if (static_cast<int>(threadIdx.x) >= off) incl += o;
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) gst[threadIdx.x * 8 + i] = incl - sum + local[i];
-        if (threadIdx.x == 31) gst[256] = incl;
+    for (int j = 0; j < kScanPer; ++j) {
+        const int i = tid + j * kPrepThreads;
+        s_start[i] = i < nkeys ? count2[i] : 0;
     }
     __syncthreads();
-    const int c0 = blockIdx.x;
-    if (c0 == 0) {
-        gstart[threadIdx.x] = gst[threadIdx.x];
-        if (threadIdx.x == 0) gstart[256] = gst[256];
+    // exclusive prefix sum: kScanPer consecutive keys per thread
+    int local[kScanPer], sum = 0;
+#pragma unroll
+    for (int j = 0; j < kScanPer; ++j) {
+        local[j] = sum;
+        sum += s_start[tid * kScanPer + j];
     }
-    const int C = meta->C;
-    if (meta->two_level == 0) {
-        if (c0 == 0) start2[threadIdx.x] = gst[threadIdx.x];
-        return;
-    }
-    if (c0 >= C) return;
-    // exclusive prefix over the C + 1 <= 128 keys of first class c0
-    const int t = threadIdx.x;
-    const int mine = t <= C ? count2[c0 * kKeyStride + t] : 0;
-    int incl = mine;
+    int incl = sum;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
         const int o = __shfl_up_sync(kFullWarp, incl, off);
-        if ((t & 31) >= off) incl += o;
+        if (lane >= off) incl += o;
     }
-    if ((t & 31) == 31) wsum[t >> 5] = incl;
+    if (lane == 31) wsum[warp] = incl;
     __syncthreads();
-    int before = 0;
-    for (int w = 0; w < (t >> 5); ++w) before += wsum[w];
-    if (t <= C) start2[c0 * kKeyStride + t] = gst[c0] + before + incl - mine;
-}
-
-// Bucket keys are counted and ranked per block of kSortTokens tokens in shared memory
-// (one counter per key), so that global memory sees one atomic per block and key instead
-// of one per token: tokens that start with a space are a third of a BPE vocabulary and
-// would otherwise all hit the same few counters.
-constexpr int kSortThreads = 1024;
-constexpr int kSortTokens = kSortThreads;
-
-__global__ void __launch_bounds__(kSortThreads)
-count_keys(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vocab_offsets,
-           int64_t vocab_nbytes, int32_t N, int32_t eos_id, const IndexMeta* __restrict__ meta,
-           const uint8_t* __restrict__ cls, int32_t* __restrict__ gcount,
-           int32_t* __restrict__ count2, uint32_t* __restrict__ planes, int32_t* status) {
-    extern __shared__ int s_cnt[];  // [kKeys]
-    __shared__ int hist[256];
-    __shared__ uint8_t s_cls[256];
-    if (threadIdx.x < 256) {
-        hist[threadIdx.x] = 0;
-        s_cls[threadIdx.x] = cls[threadIdx.x];
+    int before = 0, total = 0;
+    for (int w = 0; w < kPrepThreads / 32; ++w) {
+        if (w < warp) before += wsum[w];
+        total += wsum[w];
     }
-    const bool two = meta->two_level != 0;
-    const int nkeys = two ? kKeys : 256;
-    for (int i = threadIdx.x; i < nkeys; i += kSortThreads) s_cnt[i] = 0;
-    // bucket walk: plane c holds the bits of the one-byte tokens of class c; the block owns
-    // 32 words of every plane and clears them first
-    const int W = (N + 31) / 32;
-    if (planes != nullptr) {
-        const int C = meta->C;
-        for (int i = threadIdx.x; i < C * 32; i += kSortThreads) {
-            const int word = blockIdx.x * 32 + (i & 31);
-            if (word < W) planes[static_cast<size_t>(i >> 5) * W + word] = 0;
+#pragma unroll
+    for (int j = 0; j < kScanPer; ++j) s_start[tid * kScanPer + j] = before + incl - sum + local[j];
+    __syncthreads();
+    if (blockIdx.x == 0) {
+        for (int i = tid; i < nkeys; i += kPrepThreads) start2[i] = s_start[i];
+        if (tid <= 256) {
+            int g = total;
+            if (two) {
+                if (tid < kKeyStride) g = s_start[tid * kKeyStride];
+            } else if (tid < 256) {
+                g = s_start[tid];
+            }
+            gstart[tid] = g;
         }
     }
-    __syncthreads();
-    bool bad = false;
-    const int64_t v = static_cast<int64_t>(blockIdx.x) * kSortTokens + threadIdx.x;
-    const TokenInfo t = token_info(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, s_cls, v, &bad);
-    if (t.len > 0) {
-        atomicAdd(&hist[t.first], 1);
-        atomicAdd(&s_cnt[bucket_key(two, t.first, t.second_key)], 1);
-    }
-    if (planes != nullptr) {
-        const bool one = t.len == 1;
-        const uint32_t peers = __match_any_sync(kFullWarp, one ? t.first : 0xFFFF);
-        if (one && (threadIdx.x & 31) == __ffs(peers) - 1)
-            planes[static_cast<size_t>(t.first) * W + (v >> 5)] = peers;
-    }
-    if (__syncthreads_or(bad) && threadIdx.x == 0) raise_flag(status, FSM_FLAG_OFFSETS);
-    for (int i = threadIdx.x; i < nkeys; i += kSortThreads)
-        if (s_cnt[i] > 0) atomicAdd(&count2[i], s_cnt[i]);
-    if (threadIdx.x < 256 && hist[threadIdx.x] > 0) atomicAdd(&gcount[threadIdx.x], hist[threadIdx.x]);
-}
-
-__global__ void __launch_bounds__(kSortThreads)
-sort_tokens(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vocab_offsets,
-            int64_t vocab_nbytes, int32_t N, int32_t eos_id, const IndexMeta* __restrict__ meta,
-            const uint8_t* __restrict__ cls, const int32_t* __restrict__ start2,
-            int32_t* __restrict__ cursor2, uint4* __restrict__ srec, int32_t* __restrict__ sid) {
-    extern __shared__ int s_cnt[];  // [kKeys] count, then the block's base position per key
-    __shared__ uint8_t s_cls[256];
-    if (threadIdx.x < 256) s_cls[threadIdx.x] = cls[threadIdx.x];
-    const bool two = meta->two_level != 0;
-    const int nkeys = two ? kKeys : 256;
-    for (int i = threadIdx.x; i < nkeys; i += kSortThreads) s_cnt[i] = 0;
-    __syncthreads();
-    bool bad = false;
-    const int64_t v = static_cast<int64_t>(blockIdx.x) * kSortTokens + threadIdx.x;
-    const TokenInfo t = token_info(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, s_cls, v, &bad);
-    const int key = t.len > 0 ? bucket_key(two, t.first, t.second_key) : 0;
-    int rank = 0;
-    if (t.len > 0) rank = atomicAdd(&s_cnt[key], 1);
-    __syncthreads();
-    // one global atomic per key present in the block reserves its positions
-    for (int i = threadIdx.x; i < nkeys; i += kSortThreads) {
-        const int c = s_cnt[i];
-        if (c > 0) s_cnt[i] = start2[i] + atomicAdd(&cursor2[i], c);
-    }
-    __syncthreads();
-    if (t.len > 0) {
-        const int pos = s_cnt[key] + rank;
-        uint32_t w[4] = {static_cast<uint32_t>(t.len), 0, 0, 0};
-        const int nb = min(t.len, kInlineBytes);
-        uint8_t raw[kInlineBytes];
+    const int nchunks = (N + kPrepTokens - 1) / kPrepTokens;
+    for (int chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
+        __syncthreads();  // the previous pass is done with s_cnt
+        for (int i = tid; i < nkeys; i += kPrepThreads) s_cnt[i] = 0;
+        __syncthreads();
+        bool bad = false;
+        const int64_t v = static_cast<int64_t>(chunk) * kPrepTokens + tid;
+        const bool first = chunk == static_cast<int>(blockIdx.x);
+        const TokenRaw raw = first ? raw_first
+                                   : token_raw(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, v, &bad);
+        const TokenInfo t = token_classify(raw, s_cls);
+        const int key = t.len > 0 ? bucket_key(two, t.first, t.second_key) : 0;
+        int rank = 0;
+        if (t.len > 0) rank = atomicAdd(&s_cnt[key], 1);
+        uint8_t bytes[kInlineBytes];
 #pragma unroll
-        for (int i = 1; i < kInlineBytes; ++i)  // independent loads, issued together
-            raw[i] = i < nb ? vocab_bytes[t.start + i] : 0;
+        for (int i = 1; i < kInlineBytes; ++i) {  // independent loads, issued together
+            if (first)
+                bytes[i] = bytes_first[i];
+            else
+                bytes[i] = i < t.len ? vocab_bytes[t.start + i] : 0;
+        }
+        __syncthreads();
+        // one global atomic per key present in the pass reserves its positions; a thread
+        // issues all of its atomics before it uses the first result
+        {
+            int cnt[kScanPer], base[kScanPer];
 #pragma unroll
-        for (int i = 1; i < kInlineBytes; ++i)
-            if (i < nb) w[i >> 2] |= static_cast<uint32_t>(s_cls[raw[i]]) << ((i & 3) * 8);
-        srec[pos] = make_uint4(w[0], w[1], w[2], w[3]);
-        sid[pos] = static_cast<int32_t>(v);
+            for (int j = 0; j < kScanPer; ++j) {
+                const int i = tid + j * kPrepThreads;
+                cnt[j] = i < nkeys ? s_cnt[i] : 0;
+            }
+#pragma unroll
+            for (int j = 0; j < kScanPer; ++j) {
+                base[j] = 0;
+                if (cnt[j] > 0) base[j] = atomicAdd(&cursor2[tid + j * kPrepThreads], cnt[j]);
+            }
+#pragma unroll
+            for (int j = 0; j < kScanPer; ++j) {
+                const int i = tid + j * kPrepThreads;
+                if (cnt[j] > 0) s_cnt[i] = s_start[i] + base[j];
+            }
+        }
+        __syncthreads();
+        if (t.len > 0) {
+            const int pos = s_cnt[key] + rank;
+            uint32_t w[4] = {static_cast<uint32_t>(t.len), 0, 0, 0};
+            const int nb = min(t.len, kInlineBytes);
+#pragma unroll
+            for (int i = 1; i < kInlineBytes; ++i)
+                if (i < nb) w[i >> 2] |= static_cast<uint32_t>(s_cls[bytes[i]]) << ((i & 3) * 8);
+            srec[pos] = make_uint4(w[0], w[1], w[2], w[3]);
+            sid[pos] = static_cast<int32_t>(v);
+        }
     }
 }
 

@@ -408,7 +408,6 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
     __shared__ int32_t s_gstart[260];
     __shared__ int s_ctrs[8];      // two sets of row counters (see SurvivorSink::ctrs)
     __shared__ int s_next_row[2];
-
     if (p.meta->any_bad != 0) {
         raw_rows<OutT, HAS_OUT>(p);
         return;
@@ -536,10 +535,9 @@ cudaError_t launch_sparse(const WalkParams& p, void* scratch, int grid, cudaStre
                                          static_cast<int>(p.smem_cap));
     if (e != cudaSuccess) return e;
     // what is left after staging, counters and the descriptor list may hold the table
-    kernel<<<grid, kWalkThreads, p.smem_cap, stream>>>(
-        p, static_cast<typename Entry<TabT>::type*>(scratch),
-        static_cast<uint32_t>(p.smem_cap - table_off));
-    return cudaGetLastError();
+    return launch_on(kernel, dim3(grid), dim3(kWalkThreads), p.smem_cap, stream, p,
+                             static_cast<typename Entry<TabT>::type*>(scratch),
+                             static_cast<uint32_t>(p.smem_cap - table_off));
 }
 
 template <typename TabT>
