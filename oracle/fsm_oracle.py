@@ -21,7 +21,7 @@ def build(force: bool = False) -> str:
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
         tmp = _LIB + f".tmp{os.getpid()}"
         subprocess.check_call(["gcc", "-O2", "-fopenmp", "-std=c11", "-Wall", "-Wextra", "-shared",
-                               "-fPIC", "-o", tmp, _SRC])
+                               "-fPIC", "-ffp-contract=off", "-o", tmp, _SRC, "-lm"])
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -36,6 +36,15 @@ def _load():
         lib.oracle_index_build.restype = ctypes.c_int
         lib.oracle_mask_step.argtypes = [p, p, i32, i64, p, p, p, p, p, i32, i32, i32, i32, i32, i32]
         lib.oracle_mask_step.restype = ctypes.c_int
+        lib.oracle_sample_step.argtypes = [p, p, i32, i64, p, p, p, p, p, i32, i32, i32, i32, i32,
+                                           ctypes.c_float, ctypes.c_uint64, ctypes.c_uint64, i32]
+        lib.oracle_sample_step.restype = ctypes.c_int
+        lib.oracle_philox4x32_10.argtypes = [p, p, p]
+        lib.oracle_philox4x32_10.restype = None
+        lib.oracle_ln_f32.argtypes = [ctypes.c_float]
+        lib.oracle_ln_f32.restype = ctypes.c_float
+        lib.oracle_gumbel_f32.argtypes = [ctypes.c_uint32]
+        lib.oracle_gumbel_f32.restype = ctypes.c_float
         _lib = lib
     return _lib
 
@@ -106,3 +115,50 @@ def mask_step(logits, states, finished, allowed_mask, next_state, dead_state, eo
     if rc != 0:
         raise ValueError(f"oracle_mask_step failed with {rc}")
     return tokens, out
+
+
+def sample_step(logits, states, finished, allowed_mask, next_state, dead_state, eos_id,
+                inv_temperature, seed, draw, write_logits=True, threads=1):
+    """One masked sampling step (categorical draw by Gumbel-max with Philox bits).
+    Same conventions as ``mask_step``; ``seed`` and ``draw`` are 64-bit integers."""
+    assert logits.ndim == 2 and logits.flags.c_contiguous
+    if logits.dtype == np.float32:
+        dtype = 0
+    elif logits.dtype == np.uint16:
+        dtype = 1
+    else:
+        raise TypeError("logits must be float32 or uint16 (bf16 bits)")
+    B, N = logits.shape
+    allowed_mask = _c(allowed_mask, np.uint32)
+    next_state = _c(next_state, np.int32)
+    Q = allowed_mask.shape[0]
+    assert allowed_mask.shape == (Q, (N + 31) // 32) and next_state.shape == (Q, N)
+    assert states.dtype == np.int32 and finished.dtype == np.uint8
+    out = np.empty_like(logits) if write_logits else None
+    if out is not None:
+        out[...] = logits
+    tokens = np.empty(B, dtype=np.int32)
+    rc = _load().oracle_sample_step(_ptr(logits), _ptr(out), dtype, N, _ptr(states), _ptr(finished),
+                                    _ptr(tokens), _ptr(allowed_mask), _ptr(next_state),
+                                    Q, N, B, dead_state, eos_id, float(np.float32(inv_temperature)),
+                                    seed & 0xFFFFFFFFFFFFFFFF, draw & 0xFFFFFFFFFFFFFFFF, threads)
+    if rc != 0:
+        raise ValueError(f"oracle_sample_step failed with {rc}")
+    return tokens, out
+
+
+def philox4x32_10(ctr, key):
+    """Philox4x32-10 block: ``ctr`` four and ``key`` two 32-bit words -> four words."""
+    c = np.asarray(ctr, dtype=np.uint32).copy()
+    k = np.asarray(key, dtype=np.uint32).copy()
+    out = np.zeros(4, dtype=np.uint32)
+    _load().oracle_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return [int(x) for x in out]
+
+
+def ln_f32(x: float) -> float:
+    return float(_load().oracle_ln_f32(float(np.float32(x))))
+
+
+def gumbel_f32(bits: int) -> float:
+    return float(_load().oracle_gumbel_f32(bits & 0xFFFFFFFF))
