@@ -194,6 +194,38 @@ int guided_mask_step(const void* logits_in, void* logits_out, int32_t logits_dty
                      void* cuda_stream);
 
 /*
+ * One step of guided decoding with the categorical draw of paper Algorithm 2
+ * ("Sample s ~ Categorical(alpha~)"): as guided_mask_step, except that the token is
+ * drawn from the softmax of the masked logits divided by the temperature
+ * (Section 2.1 calls this multinomial sampling; the paper's runs use temperature 0.1).
+ *
+ * The draw is the Gumbel-max form of that distribution, so that the step is a pure
+ * function of its arguments:
+ *   tok = argmax over v in sigma(q) of fma(logit[v], inv_temperature, G(v)), ties to
+ *         the lowest id, with G(v) = -ln(-ln(u(v))) a standard Gumbel variate;
+ *   u(v) = (2*(r >> 9) + 1) * 2^-24 with r the 32-bit word v % 4 of
+ *         Philox4x32-10(key = (seed low, seed high),
+ *                       counter = (v / 4, batch row, draw low, draw high))
+ *         (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3",
+ *         SC'11);
+ *   ln is evaluated in fp32 with explicitly rounded operations: x = m 2^e, m in
+ *         (sqrt(1/2), sqrt(2)], s = (m-1)/(m+1), ln m = 2s(1 + s^2/3 + s^4/5 + s^6/7 +
+ *         s^8/9) by Horner's rule with fused multiply-adds, ln x = fma(e, ln 2, ln m).
+ * Logits are widened to fp32 exactly.  Rows, masking, EOS, stuck rows, finished rows,
+ * the state update and every other argument are as in guided_mask_step.
+ *
+ *   inv_temperature  1 / temperature as fp32, > 0 and finite (FSM_ERR_RANGE otherwise).
+ *   seed, draw       64-bit key and draw number: use a new `draw` for every step (the
+ *                    step index), the same `seed` for a sequence of steps.
+ */
+int guided_sample_step(const void* logits_in, void* logits_out, int32_t logits_dtype,
+                       int64_t row_stride, int32_t* states, uint8_t* finished,
+                       int32_t* tokens_out, const uint32_t* allowed_mask,
+                       const void* next_state, int32_t state_dtype, int32_t Q, int32_t N,
+                       int32_t B, int32_t dead_state, int32_t eos_id, float inv_temperature,
+                       uint64_t seed, uint64_t draw, int32_t* status_word, void* cuda_stream);
+
+/*
  * Tuning and test hooks (no counterpart in the paper).  Sets a process-wide knob
  * and returns the previous value, or FSM_ERR_RANGE for an unknown key.  Not
  * thread-safe against concurrent library calls.

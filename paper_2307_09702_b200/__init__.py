@@ -1,4 +1,4 @@
-"""fsmguide: FSM vocabulary indexing and masked greedy decoding on NVIDIA B200.
+"""fsmguide: FSM vocabulary indexing and masked greedy / sampled decoding on NVIDIA B200.
 
 The work is done by hand-written CUDA kernels behind a C ABI
 (``include/fsmguide.h``, built into ``libfsmguide.so``); this package is the thin
@@ -8,11 +8,11 @@ built library raises.
 from .binding import (FSM_LOGITS_BF16, FSM_LOGITS_F32, FSM_STATE_I32, FSM_STATE_U16, FsmError,
                       GuidedIndex, fsm_debug_set, fsm_device_check, fsm_index_build,
                       fsm_index_build_rows, fsm_index_build_static, fsm_index_workspace_bytes, fsm_profile_read, fsm_status_string,
-                      guided_mask_step, lib, library_path)
+                      guided_mask_step, guided_sample_step, lib, library_path)
 
 __all__ = [
     "FSM_LOGITS_BF16", "FSM_LOGITS_F32", "FSM_STATE_I32", "FSM_STATE_U16", "FsmError",
     "GuidedIndex", "fsm_debug_set", "fsm_device_check", "fsm_index_build",
     "fsm_index_build_rows", "fsm_index_build_static", "fsm_index_workspace_bytes", "fsm_profile_read", "fsm_status_string",
-    "guided_mask_step", "lib", "library_path",
+    "guided_mask_step", "guided_sample_step", "lib", "library_path",
 ]

@@ -66,6 +66,9 @@ def lib() -> ctypes.CDLL:
         L.guided_mask_step.argtypes = [vp, vp, i32, i64, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32,
                                        i32, vp, vp]
         L.guided_mask_step.restype = ctypes.c_int
+        L.guided_sample_step.argtypes = [vp, vp, i32, i64, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32,
+                                         i32, ctypes.c_float, ctypes.c_uint64, ctypes.c_uint64, vp, vp]
+        L.guided_sample_step.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -149,6 +152,17 @@ def guided_mask_step(logits_in, logits_out, logits_dtype, row_stride, states, fi
                                   _ptr(status_word), _stream(stream))
 
 
+def guided_sample_step(logits_in, logits_out, logits_dtype, row_stride, states, finished, tokens_out,
+                       allowed_mask, next_state, state_dtype, Q, N, B, dead_state, eos_id,
+                       inv_temperature, seed, draw, status_word=None, stream=None) -> int:
+    return lib().guided_sample_step(_ptr(logits_in), _ptr(logits_out), logits_dtype, row_stride,
+                                    _ptr(states), _ptr(finished), _ptr(tokens_out),
+                                    _ptr(allowed_mask), _ptr(next_state), state_dtype, Q, N, B,
+                                    dead_state, eos_id, inv_temperature,
+                                    seed & 0xFFFFFFFFFFFFFFFF, draw & 0xFFFFFFFFFFFFFFFF,
+                                    _ptr(status_word), _stream(stream))
+
+
 class GuidedIndex:
     """Holds the device buffers of one vocabulary index and forwards to the C ABI.
 
@@ -203,3 +217,20 @@ class GuidedIndex:
                               logits.shape[0], self.dead_state, self.eos_id, self.status, stream)
         if rc != 0:
             raise FsmError(rc, "guided_mask_step")
+
+    def sample(self, logits, states, finished, tokens_out, inv_temperature, seed, draw,
+               logits_out="inplace", stream=None):
+        """One masked sampling step (categorical draw) on ``logits`` [B, >=N]."""
+        if logits.dtype == torch.float32:
+            ldt = FSM_LOGITS_F32
+        elif logits.dtype == torch.bfloat16:
+            ldt = FSM_LOGITS_BF16
+        else:
+            raise TypeError("logits must be float32 or bfloat16")
+        out = logits if isinstance(logits_out, str) else logits_out
+        rc = guided_sample_step(logits, out, ldt, logits.stride(0), states, finished, tokens_out,
+                                self.allowed_mask, self.next_state, self.state_dtype, self.Q, self.N,
+                                logits.shape[0], self.dead_state, self.eos_id, inv_temperature, seed,
+                                draw, self.status, stream)
+        if rc != 0:
+            raise FsmError(rc, "guided_sample_step")

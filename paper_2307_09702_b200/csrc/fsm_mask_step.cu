@@ -1,4 +1,5 @@
-// Masked greedy decode step (paper Algorithm 2 with argmax selection) for sm_100a.
+// Masked decode step (paper Algorithm 2) for sm_100a: greedy selection (Section 2.1) or
+// the categorical draw of Algorithm 2 itself, as a Gumbel-max over the allowed tokens.
 //
 // One thread-block cluster of `k` CTAs owns one logits row.  Each thread streams
 // 32-byte vectors of the row: it first reads the vector's bits of the allowed-token
@@ -33,6 +34,9 @@ struct StepParams {
     int32_t state_u16;
     int32_t Q, N, W, B, dead, eos_id, k;
     int32_t* status;
+    // sampling
+    float inv_temperature;
+    uint32_t seed_lo, seed_hi, draw_lo, draw_hi;
 };
 
 struct Best {
@@ -116,7 +120,82 @@ __device__ __forceinline__ int locate(const uint32_t (&w)[NW], uint32_t bits, fl
     return pos;
 }
 
-template <typename T, bool WRITE>
+// ---------------------------------------------------------------------------------------
+// Categorical draw (Algorithm 2): argmax over the allowed tokens of
+// logit / temperature + G with G a standard Gumbel variate.  The random bits come from
+// Philox4x32-10 (Salmon et al., SC'11) with key = seed and counter = (token id / 4, batch
+// row, draw number); token v uses output word v % 4.  Every floating-point step is an
+// explicitly rounded fp32 operation, so the result does not depend on compiler flags.
+__device__ __forceinline__ uint32_t philox_word(uint32_t v, uint32_t row, const StepParams& p) {
+    uint32_t c0 = v >> 2, c1 = row, c2 = p.draw_lo, c3 = p.draw_hi;
+    uint32_t k0 = p.seed_lo, k1 = p.seed_hi;
+#pragma unroll
+    for (int round = 0; round < 10; ++round) {
+        const unsigned long long a = static_cast<unsigned long long>(c0) * 0xD2511F53ull;
+        const unsigned long long b = static_cast<unsigned long long>(c2) * 0xCD9E8D57ull;
+        c0 = static_cast<uint32_t>(b >> 32) ^ c1 ^ k0;
+        c2 = static_cast<uint32_t>(a >> 32) ^ c3 ^ k1;
+        c1 = static_cast<uint32_t>(b);
+        c3 = static_cast<uint32_t>(a);
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    const uint32_t sel = v & 3u;
+    return sel == 0 ? c0 : sel == 1 ? c1 : sel == 2 ? c2 : c3;
+}
+
+// ln x of a positive normal x: x = m 2^e with m in (sqrt(1/2), sqrt(2)], s = (m-1)/(m+1),
+// ln m = 2 s (1 + s^2/3 + s^4/5 + s^6/7 + s^8/9) by Horner's rule.
+__device__ __forceinline__ float ln_rn(float x) {
+    const uint32_t b = __float_as_uint(x);
+    int e = static_cast<int>(b >> 23) - 127;
+    float m = __uint_as_float((b & 0x007FFFFFu) | 0x3F800000u);
+    if (m > 1.41421354f) {
+        m = __fmul_rn(m, 0.5f);
+        e += 1;
+    }
+    const float s = __fdiv_rn(__fadd_rn(m, -1.0f), __fadd_rn(m, 1.0f));
+    const float z = __fmul_rn(s, s);
+    float t = __fmaf_rn(z, 1.0f / 9.0f, 1.0f / 7.0f);
+    t = __fmaf_rn(z, t, 1.0f / 5.0f);
+    t = __fmaf_rn(z, t, 1.0f / 3.0f);
+    t = __fmaf_rn(z, t, 1.0f);
+    return __fmaf_rn(static_cast<float>(e), 0.693147182f, __fmul_rn(__fadd_rn(s, s), t));
+}
+
+__device__ __forceinline__ float gumbel_score(float x, uint32_t v, uint32_t row, const StepParams& p) {
+    const uint32_t bits = philox_word(v, row, p);
+    // u: an odd multiple of 2^-24 strictly inside (0, 1)
+    const float u = __fmul_rn(static_cast<float>(2u * (bits >> 9) + 1u), 5.9604644775390625e-08f);
+    const float y = -ln_rn(u);
+    return __fmaf_rn(x, p.inv_temperature, -ln_rn(y));
+}
+
+// Masks one vector of NW words in place and folds the scores of its allowed entries into
+// the thread's best (score, id).  Ids only grow within a thread, so a strict comparison
+// keeps the lowest id among equal scores.
+template <typename T, int NW>
+__device__ __forceinline__ void process_sample(uint32_t (&w)[NW], uint32_t bits, int first_id,
+                                               uint32_t row, const StepParams& p, Best& best) {
+    constexpr int PW = Elem<T>::kPerWord;
+    uint32_t todo = bits;
+    while (todo) {
+        const int j = __ffs(todo) - 1;
+        todo &= todo - 1;
+        uint32_t word = w[0];
+#pragma unroll
+        for (int i = 1; i < NW; ++i) word = (j / PW == i) ? w[i] : word;
+        const float score = gumbel_score(Elem<T>::get(word, j % PW), first_id + j, row, p);
+        if (best.idx == kNone || score > best.val) {
+            best.val = score;
+            best.idx = first_id + j;
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < NW; ++i) w[i] = Elem<T>::select(w[i], (bits >> (i * PW)) & ((1u << PW) - 1u));
+}
+
+template <typename T, bool WRITE, bool SAMPLE>
 __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
     cg::cluster_group cluster = cg::this_cluster();
     __shared__ Best warp_best[kStepWarps];
@@ -142,6 +221,7 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
     const bool wide = ((reinterpret_cast<uintptr_t>(in) | (WRITE ? reinterpret_cast<uintptr_t>(out) : 0)) & 31) == 0;
 
     ThreadBest tb{__int_as_float(0x7FC00000), -1, 0u};
+    Best best{0.0f, kNone};
     const int tid = rank * kStepThreads + threadIdx.x;
     const int nthreads = k * kStepThreads;
 
@@ -174,7 +254,10 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
                     const int vi = g0 + (h + u) * nthreads;
                     if (vi < nvec) {
                         if (bits[h + u] != 0) {
-                            process<T, 8>(v[u].w, bits[h + u], vi, tb);
+                            if (SAMPLE)
+                                process_sample<T, 8>(v[u].w, bits[h + u], vi * EPV, row, p, best);
+                            else
+                                process<T, 8>(v[u].w, bits[h + u], vi, tb);
                         } else {
 #pragma unroll
                             for (int i = 0; i < 8; ++i) v[u].w[i] = Elem<T>::kNegInfWord;
@@ -194,7 +277,10 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
             if (bits != 0) {
                 const uint4 v = *reinterpret_cast<const uint4*>(in + e0);
                 w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
-                process<T, 4>(w, bits, vi, tb);
+                if (SAMPLE)
+                    process_sample<T, 4>(w, bits, e0, row, p, best);
+                else
+                    process<T, 4>(w, bits, vi, tb);
             } else {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) w[i] = Elem<T>::kNegInfWord;
@@ -206,8 +292,7 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
     // Position of the thread's maximum: re-read the winning vector (the allowed entries
     // are unchanged by the masking, wherever it was written) and take the lowest
     // allowed position that holds the value.
-    Best best{0.0f, kNone};
-    if (tb.vec >= 0) {
+    if (!SAMPLE && tb.vec >= 0) {
         const T* src = (WRITE ? static_cast<const T*>(out) : in);
         best.val = tb.val;
         if (wide) {
@@ -226,8 +311,9 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
             const bool allowed = (live & (mrow[e >> 5] >> (e & 31)) & 1u) != 0;
             const T raw = in[e];
             if (allowed) {
-                const float x = sizeof(T) == 4 ? __uint_as_float(static_cast<uint32_t>(raw))
-                                               : __uint_as_float(static_cast<uint32_t>(raw) << 16);
+                float x = sizeof(T) == 4 ? __uint_as_float(static_cast<uint32_t>(raw))
+                                         : __uint_as_float(static_cast<uint32_t>(raw) << 16);
+                if (SAMPLE) x = gumbel_score(x, e, row, p);
                 if (best.idx == kNone || x > best.val) {  // tail ids exceed every vector id
                     best.val = x;
                     best.idx = e;
@@ -277,7 +363,7 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
     }
 }
 
-template <typename T, bool WRITE>
+template <typename T, bool WRITE, bool SAMPLE>
 cudaError_t launch(const StepParams& p, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(p.B) * p.k, 1, 1);
@@ -291,18 +377,19 @@ cudaError_t launch(const StepParams& p, cudaStream_t stream) {
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, mask_step<T, WRITE>, p);
+    return cudaLaunchKernelEx(&cfg, mask_step<T, WRITE, SAMPLE>, p);
 }
 
 }  // namespace
 }  // namespace fsm
 
-extern "C" int guided_mask_step(const void* logits_in, void* logits_out, int32_t logits_dtype,
-                                int64_t row_stride, int32_t* states, uint8_t* finished,
-                                int32_t* tokens_out, const uint32_t* allowed_mask,
-                                const void* next_state, int32_t state_dtype, int32_t Q, int32_t N,
-                                int32_t B, int32_t dead_state, int32_t eos_id,
-                                int32_t* status_word, void* cuda_stream) {
+namespace {
+int step_impl(const void* logits_in, void* logits_out, int32_t logits_dtype, int64_t row_stride,
+              int32_t* states, uint8_t* finished, int32_t* tokens_out,
+              const uint32_t* allowed_mask, const void* next_state, int32_t state_dtype, int32_t Q,
+              int32_t N, int32_t B, int32_t dead_state, int32_t eos_id, bool sample,
+              float inv_temperature, uint64_t seed, uint64_t draw, int32_t* status_word,
+              void* cuda_stream) {
     using namespace fsm;
     if (Q <= 0 || N <= 0 || B < 0 || row_stride < N) return FSM_ERR_SHAPE;
     if (!logits_in || !states || !finished || !tokens_out || !allowed_mask || !next_state)
@@ -355,12 +442,48 @@ extern "C" int guided_mask_step(const void* logits_in, void* logits_out, int32_t
     p.eos_id = eos_id;
     p.k = k;
     p.status = status_word;
+    p.inv_temperature = inv_temperature;
+    p.seed_lo = static_cast<uint32_t>(seed);
+    p.seed_hi = static_cast<uint32_t>(seed >> 32);
+    p.draw_lo = static_cast<uint32_t>(draw);
+    p.draw_hi = static_cast<uint32_t>(draw >> 32);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e;
     const bool write = logits_out != nullptr;
-    if (logits_dtype == FSM_LOGITS_F32)
-        e = write ? launch<uint32_t, true>(p, stream) : launch<uint32_t, false>(p, stream);
-    else
-        e = write ? launch<uint16_t, true>(p, stream) : launch<uint16_t, false>(p, stream);
+    if (sample) {
+        if (logits_dtype == FSM_LOGITS_F32)
+            e = write ? launch<uint32_t, true, true>(p, stream) : launch<uint32_t, false, true>(p, stream);
+        else
+            e = write ? launch<uint16_t, true, true>(p, stream) : launch<uint16_t, false, true>(p, stream);
+    } else if (logits_dtype == FSM_LOGITS_F32) {
+        e = write ? launch<uint32_t, true, false>(p, stream) : launch<uint32_t, false, false>(p, stream);
+    } else {
+        e = write ? launch<uint16_t, true, false>(p, stream) : launch<uint16_t, false, false>(p, stream);
+    }
     return e == cudaSuccess ? FSM_OK : FSM_ERR_CUDA;
+}
+}  // namespace
+
+extern "C" int guided_mask_step(const void* logits_in, void* logits_out, int32_t logits_dtype,
+                                int64_t row_stride, int32_t* states, uint8_t* finished,
+                                int32_t* tokens_out, const uint32_t* allowed_mask,
+                                const void* next_state, int32_t state_dtype, int32_t Q, int32_t N,
+                                int32_t B, int32_t dead_state, int32_t eos_id,
+                                int32_t* status_word, void* cuda_stream) {
+    return step_impl(logits_in, logits_out, logits_dtype, row_stride, states, finished, tokens_out,
+                     allowed_mask, next_state, state_dtype, Q, N, B, dead_state, eos_id, false, 1.0f,
+                     0, 0, status_word, cuda_stream);
+}
+
+extern "C" int guided_sample_step(const void* logits_in, void* logits_out, int32_t logits_dtype,
+                                  int64_t row_stride, int32_t* states, uint8_t* finished,
+                                  int32_t* tokens_out, const uint32_t* allowed_mask,
+                                  const void* next_state, int32_t state_dtype, int32_t Q,
+                                  int32_t N, int32_t B, int32_t dead_state, int32_t eos_id,
+                                  float inv_temperature, uint64_t seed, uint64_t draw,
+                                  int32_t* status_word, void* cuda_stream) {
+    if (!(inv_temperature > 0.0f) || !(inv_temperature < 3.0e38f)) return FSM_ERR_RANGE;
+    return step_impl(logits_in, logits_out, logits_dtype, row_stride, states, finished, tokens_out,
+                     allowed_mask, next_state, state_dtype, Q, N, B, dead_state, eos_id, true,
+                     inv_temperature, seed, draw, status_word, cuda_stream);
 }

@@ -1,5 +1,6 @@
-"""GPU parity of guided_mask_step against the CPU oracle: masked logits, chosen
-tokens, states and finished flags are compared bit for bit (tolerance 0)."""
+"""GPU parity of guided_mask_step and guided_sample_step against the CPU oracle:
+masked logits, chosen tokens, states and finished flags are compared bit for bit
+(tolerance 0; the sampled token is a pure function of logits, seed and draw number)."""
 import numpy as np
 import pytest
 import torch
@@ -32,7 +33,9 @@ def random_index(rng, Q, N, allowed_frac=0.25):
     return np.ascontiguousarray(mask), nxt
 
 
-def run_case(rng, Q, N, B, dtype, mode, k=0, stride_pad=0, state_dtype=0, eos=5, coarse=True):
+def run_case(rng, Q, N, B, dtype, mode, k=0, stride_pad=0, state_dtype=0, eos=5, coarse=True,
+             sample=None):
+    """``sample`` = (inv_temperature, seed, draw) runs the categorical draw instead of argmax."""
     mask, nxt = random_index(rng, Q, N)
     mask[3] = 0
     x = rng.standard_normal((B, N)).astype(np.float32) * 2
@@ -51,8 +54,13 @@ def run_case(rng, Q, N, B, dtype, mode, k=0, stride_pad=0, state_dtype=0, eos=5,
         x[6, eos] = 1000.0
     host_logits = f32_to_bf16_bits(x) if dtype == "bf16" else x
     st_o, fin_o = states.copy(), finished.copy()
-    tok_o, out_o = fsm_oracle.mask_step(host_logits, st_o, fin_o, mask, nxt, Q - 1, eos,
-                                        write_logits=(mode != "select"), threads=THREADS)
+    if sample is None:
+        tok_o, out_o = fsm_oracle.mask_step(host_logits, st_o, fin_o, mask, nxt, Q - 1, eos,
+                                            write_logits=(mode != "select"), threads=THREADS)
+    else:
+        tok_o, out_o = fsm_oracle.sample_step(host_logits, st_o, fin_o, mask, nxt, Q - 1, eos,
+                                              sample[0], sample[1], sample[2],
+                                              write_logits=(mode != "select"), threads=THREADS)
 
     dev = torch.device("cuda")
     stride = N + stride_pad
@@ -79,8 +87,13 @@ def run_case(rng, Q, N, B, dtype, mode, k=0, stride_pad=0, state_dtype=0, eos=5,
         out = None
     fg.fsm_debug_set(2, k)
     ldt = fg.FSM_LOGITS_BF16 if dtype == "bf16" else fg.FSM_LOGITS_F32
-    rc = fg.guided_mask_step(buf, out, ldt, stride, d_states, d_fin, d_tok, d_mask, d_next,
-                             state_dtype, Q, N, B, Q - 1, eos, status)
+    if sample is None:
+        rc = fg.guided_mask_step(buf, out, ldt, stride, d_states, d_fin, d_tok, d_mask, d_next,
+                                 state_dtype, Q, N, B, Q - 1, eos, status)
+    else:
+        rc = fg.guided_sample_step(buf, out, ldt, stride, d_states, d_fin, d_tok, d_mask, d_next,
+                                   state_dtype, Q, N, B, Q - 1, eos, sample[0], sample[1],
+                                   sample[2], status)
     assert rc == 0, fg.fsm_status_string(rc)
     torch.cuda.synchronize()
     assert (d_tok.cpu().numpy() == tok_o).all(), (d_tok.cpu().numpy(), tok_o)
@@ -125,6 +138,68 @@ def test_ragged_rows_and_narrow_alignment(N, pad, dtype):
         pad = pad if (N + pad) % 8 == 0 else (-N) % 8
     run_case(np.random.default_rng(N), Q=6, N=N, B=8, dtype=dtype, mode="inplace", stride_pad=pad, eos=0)
     run_case(np.random.default_rng(N), Q=6, N=N, B=8, dtype=dtype, mode="outofplace", stride_pad=pad, eos=-1)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("mode", ["inplace", "outofplace", "select"])
+def test_sample_step_modes(dtype, mode):
+    toks = [run_case(np.random.default_rng(1), Q=11, N=5000, B=9, dtype=dtype, mode=mode,
+                     sample=(1.0, 0x0123456789ABCDEF, draw)) for draw in (0, 1, 2**40 + 7)]
+    assert any((toks[0] != t).any() for t in toks[1:])      # a new draw number, a new draw
+
+
+@pytest.mark.parametrize("inv_t", [0.25, 1.0, 10.0])
+@pytest.mark.parametrize("k", [1, 2, 4, 8])
+def test_sample_step_cluster_sizes_and_temperatures(k, inv_t):
+    run_case(np.random.default_rng(k), Q=11, N=40000, B=7, dtype="bf16", mode="inplace", k=k,
+             sample=(inv_t, 99 + k, 5), coarse=False)
+    run_case(np.random.default_rng(k), Q=11, N=20000, B=7, dtype="f32", mode="select", k=k,
+             sample=(inv_t, 99 + k, 6), coarse=False)
+
+
+@pytest.mark.parametrize("N,pad", [(1, 7), (7, 1), (33, 7), (1003, 5), (4097, 7)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_sample_step_ragged_rows(N, pad, dtype):
+    if dtype == "f32":
+        pad = (-N) % 4 if (N + pad) % 4 else pad
+    else:
+        pad = pad if (N + pad) % 8 == 0 else (-N) % 8
+    run_case(np.random.default_rng(N), Q=6, N=N, B=8, dtype=dtype, mode="inplace", stride_pad=pad,
+             eos=0, sample=(2.0, 7, 3))
+
+
+def test_sample_step_rejects_bad_temperature():
+    z = torch.zeros(8, dtype=torch.int32, device="cuda")
+    x = torch.zeros((1, 8), device="cuda")
+    f = torch.zeros(1, dtype=torch.uint8, device="cuda")
+    for bad in (0.0, -1.0, float("inf"), float("nan")):
+        assert fg.guided_sample_step(x, x, fg.FSM_LOGITS_F32, 8, z, f, z, z, z, 0, 2, 8, 1, 1, -1,
+                                     bad, 1, 1) == -6
+
+
+def test_sample_workload_5_shape_steps_match_oracle():
+    """Workload 5's shape (256 x 128,256 bf16 logits, workload 3's index), temperature 0.1
+    as in the paper's runs: 3 steps in lock step with the oracle."""
+    w = make_config(5)
+    d = w.dfa
+    idx = gpu_index(d.trans, d.accept, w.vocab_bytes, w.vocab_offsets, d.dead, w.eos_id)
+    mask, nxt = mask_np(idx), next_np(idx)
+    st = start_states(w)
+    st_o, fin_o = st.copy(), np.zeros(w.B, np.uint8)
+    d_st = torch.from_numpy(st).cuda()
+    d_fin = torch.zeros(w.B, dtype=torch.uint8, device="cuda")
+    d_tok = torch.zeros(w.B, dtype=torch.int32, device="cuda")
+    g = torch.Generator(device="cuda").manual_seed(w.seed)
+    for step in range(3):
+        x = (torch.randn((w.B, w.N), generator=g, device="cuda") * w.logits_sigma).to(torch.bfloat16)
+        host = x.view(torch.int16).cpu().numpy().view(np.uint16)
+        tok_o, out_o = fsm_oracle.sample_step(host, st_o, fin_o, mask, nxt, d.dead, w.eos_id, 10.0,
+                                              w.seed, step, threads=THREADS)
+        idx.sample(x, d_st, d_fin, d_tok, 10.0, w.seed, step)
+        torch.cuda.synchronize()
+        assert (d_tok.cpu().numpy() == tok_o).all()
+        assert (d_st.cpu().numpy() == st_o).all() and (d_fin.cpu().numpy() == fin_o).all()
+        assert (x.view(torch.int16).cpu().numpy().view(np.uint16) == out_o).all()
 
 
 def test_u16_next_state_and_smooth_logits():
