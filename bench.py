@@ -10,8 +10,9 @@ B = 256 bf16 logits rows of that vocabulary, in place.
 
 Prints one JSON line.  ``value`` is (state, token) walks per second of the index
 build (Q*N per build, all ranks, divided by the build's device time inside the
-step); ``mask_step_us`` is the masked-logit step; ``ms_per_step`` is the whole
-step.  With N > 1 (torchrun) every rank runs the same-shaped workload on its own
+step); ``mask_step_us`` is the masked-logit step (``sample_step_us`` the same step with the
+categorical draw at temperature 0.1 instead of the argmax); ``ms_per_step`` is the
+whole step.  With N > 1 (torchrun) every rank runs the same-shaped workload on its own
 GPU with its own automaton seed: the path shards over independent problems and
 has no data-path collective (weak scaling).
 
@@ -40,6 +41,8 @@ SMEM_LOOKUP_BOUND = 148 * 32 * 1.965e9 / 1.157
 # (walk_sparse_config3.md, mask_step_config5.md).  Set an entry to None when the kernel
 # changes and the capture has not been redone.
 NCU_TRAFFIC = {"walk_sparse": 509_200_000, "mask_step": 66_570_000}
+# kernels of this library per timed step: hash_columns, prepare_all, sort_all, walk_sparse,
+# mask_step
 RING = 8
 
 
@@ -309,6 +312,20 @@ def run_ours(args):
     barrier()
     mask_loop_ms = m_begin.elapsed_time(m_end) / mask_loop_steps
     rows_live_end = int((fin == 0).sum().item())
+    # ---- the same loop with the categorical draw (temperature 0.1, as in the paper's runs)
+    st.copy_(st0)
+    fin.copy_(fin0)
+    for i in range(args.warmup):
+        idx.sample(ring[i % RING], st, fin, tok, 10.0, w.seed, i)
+    st.copy_(st0)
+    fin.copy_(fin0)
+    barrier()
+    m_begin.record()
+    for i in range(mask_loop_steps):
+        idx.sample(ring[i % RING], st, fin, tok, 10.0, w.seed, 1000 + i)
+    m_end.record()
+    barrier()
+    sample_ms = m_begin.elapsed_time(m_end) / mask_loop_steps
     build_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in events]))
     mask_in_step_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in events]))
     mask_ms = mask_loop_ms
@@ -378,9 +395,9 @@ def run_ours(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
 
-    total_ms, build_ms, mask_ms, mask_in_step_ms, walk_ms_mean, e2e_s, u16_ms, maskonly_ms = map(
-        allmax, (total_ms, build_ms, mask_ms, mask_in_step_ms, walk_ms_mean, e2e_s, u16_ms,
-                 maskonly_ms))
+    (total_ms, build_ms, mask_ms, mask_in_step_ms, walk_ms_mean, e2e_s, u16_ms, maskonly_ms,
+     sample_ms) = map(allmax, (total_ms, build_ms, mask_ms, mask_in_step_ms, walk_ms_mean, e2e_s,
+                               u16_ms, maskonly_ms, sample_ms))
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -399,6 +416,7 @@ def run_ours(args):
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int32", "data": "synthetic",
         "index_build_us": build_ms * 1e3, "mask_step_us": mask_ms * 1e3,
+        "sample_step_us": sample_ms * 1e3,
         "mask_step_in_step_us": mask_in_step_ms * 1e3, "walk_kernel_us": walk_ms_mean * 1e3,
         "mask_step_loop": {"steps": mask_loop_steps, "live_rows_at_end": rows_live_end,
                            "note": "mask_step_us: back-to-back decode loop over the logits ring; "
@@ -416,6 +434,13 @@ def run_ours(args):
                                "frac": mask_achieved / hbm_gbs, "peak_kind": f"of {peak_kind}",
                                "algorithmic_bytes_per_launch": mask_bytes,
                                "traffic": NCU_TRAFFIC.get("mask_step")},
+        "roofline_sample_step": {"bound": "hbm", "kernel": "mask_step (categorical draw)",
+                                 "achieved": mask_bytes / (sample_ms * 1e-3) / 1e9, "peak": hbm_gbs,
+                                 "unit": "GB/s", "frac": mask_bytes / (sample_ms * 1e-3) / 1e9 / hbm_gbs,
+                                 "peak_kind": f"of {peak_kind}",
+                                 "algorithmic_bytes_per_launch": mask_bytes, "traffic": None,
+                                 "note": "same bytes as the greedy step; the draw adds about 125 "
+                                         "integer/fp32 instructions per allowed token"},
         "index_build_modes": {
             "int32_states": {"us": build_ms * 1e3, "walks_per_s": walks / (build_ms * 1e-3),
                              "hbm_write_bound_frac": (walks * 4.125 / (build_ms * 1e-3) / 1e9) / hbm_gbs},
@@ -431,7 +456,7 @@ def run_ours(args):
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "note": "host DFA, vocabulary, logits and states copied in, tokens/states/finished "
                         "copied out, every step; the index stays on the device for its consumer"},
-        "gpu_launches": 8 * args.steps,
+        "gpu_launches": 5 * args.steps,
     }
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(w, starts)
@@ -447,8 +472,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--walk-algo", type=int, default=0, choices=[0, 1, 2],
-                    help="index walk kernel: 0 automatic, 1 dense warp-tile, 2 work-avoiding")
+    ap.add_argument("--walk-algo", type=int, default=0, choices=[0, 1, 2, 3],
+                    help="index walk: 0 automatic, 1 dense warp-tile, 2 row-wise work-avoiding, "
+                         "3 bucket walk (bitmask-only builds)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
