@@ -5,6 +5,7 @@ The work is done by hand-written CUDA kernels behind a C ABI
 Python binding.  There is no CPU fallback: importing the binding without the
 built library raises.
 """
+from .batching import stack_automata
 from .binding import (FSM_LOGITS_BF16, FSM_LOGITS_F32, FSM_STATE_I32, FSM_STATE_U16, FsmError,
                       GuidedIndex, fsm_debug_set, fsm_device_check, fsm_index_build,
                       fsm_index_build_rows, fsm_index_build_static, fsm_index_workspace_bytes, fsm_profile_read, fsm_status_string,
@@ -14,5 +15,5 @@ __all__ = [
     "FSM_LOGITS_BF16", "FSM_LOGITS_F32", "FSM_STATE_I32", "FSM_STATE_U16", "FsmError",
     "GuidedIndex", "fsm_debug_set", "fsm_device_check", "fsm_index_build",
     "fsm_index_build_rows", "fsm_index_build_static", "fsm_index_workspace_bytes", "fsm_profile_read", "fsm_status_string",
-    "guided_mask_step", "guided_sample_step", "lib", "library_path",
+    "guided_mask_step", "guided_sample_step", "lib", "library_path", "stack_automata",
 ]

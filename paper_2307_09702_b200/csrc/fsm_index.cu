@@ -156,7 +156,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     p.next = next_state;
     p.status = status_word;
     const int min_cap = sparse ? static_cast<int>(sparse_table_offset<int32_t>(N)) + 4096
-                               : kChunk * kMaxCs * 4;
+                               : (kChunk + 4) * kMaxCs * 4;
     if (cap < min_cap) cap = min_cap;
     p.smem_cap = static_cast<uint32_t>(cap) / 128 * 128;
 

@@ -31,7 +31,8 @@ constexpr int kStatesPerTask = 128;   // states scanned by one walk_buckets task
 template <typename TabT>
 __device__ __forceinline__ bool stage_table(const WalkParams& p, TabT* stab, uint64_t* bar,
                                             uint32_t table_cap, uint32_t Cs, bool& full) {
-    const uint64_t table_bytes = static_cast<uint64_t>(p.Q) * Cs * sizeof(TabT);
+    // (a bulk copy moves multiples of 16 bytes; the table's workspace has the slack)
+    const uint64_t table_bytes = (static_cast<uint64_t>(p.Q) * Cs * sizeof(TabT) + 15) / 16 * 16;
     full = table_bytes <= table_cap;
     if (!full) return true;
     if (threadIdx.x == 0) {

@@ -7,7 +7,7 @@ namespace fsm {
 namespace {
 
 constexpr int kHashBlocks = 32;
-constexpr int kMaxCs = 264;             // 256 classes + the null class, rounded up to 8
+constexpr int kMaxCs = 264;             // bound on the row stride (256 classes + the null class)
 constexpr int kWalkThreads = 1024;
 constexpr int kWalkWarps = kWalkThreads / 32;
 constexpr int kChunk = 32;              // states per warp task (dense walk)
@@ -51,6 +51,15 @@ struct Workspace {
 };
 
 inline size_t table_elem_bytes(int32_t Q) { return Q <= 65535 ? 2 : 4; }
+
+// Row stride of the compressed table in entries: room for C classes and the null class,
+// and an odd number of 32-bit words, so that the same column of 32 different rows lies
+// in 32 different shared-memory banks (lanes that hold different states and look up one
+// class do not conflict).
+template <typename TabT>
+__host__ __device__ constexpr int table_row_stride(int C) {
+    return sizeof(TabT) == 2 ? ((C + 1 + 1) / 4 * 4 + 2) : ((C + 1) | 1);
+}
 
 inline Workspace carve(void* base, int32_t Q, int32_t N) {
     Workspace w;

@@ -84,8 +84,11 @@ __global__ void __launch_bounds__(kWalkThreads, 1) walk(const WalkParams p) {
     const bool raw = p.meta->any_bad != 0;
     const uint32_t row_bytes = Cs * sizeof(TabT);
     const int nrows = p.q_end - p.q_begin;
-    const bool full = static_cast<uint64_t>(p.Q) * row_bytes <= p.smem_cap;
-    const int cap_rows = max(kChunk, static_cast<int>(p.smem_cap / row_bytes) / kChunk * kChunk);
+    // Four rows are a multiple of 16 bytes (the row stride is an odd number of words): a
+    // tile starts at a row that is a multiple of four, and its size is rounded up to 16 bytes.
+    const uint32_t tile_cap = p.smem_cap - 16;
+    const bool full = static_cast<uint64_t>(p.Q) * row_bytes <= tile_cap;
+    const int cap_rows = max(kChunk, (static_cast<int>(tile_cap / row_bytes) - 3) / kChunk * kChunk);
     const int ntiles = full ? 1 : (nrows + cap_rows - 1) / cap_rows;
     const int lane = threadIdx.x & 31;
     const int64_t wg = static_cast<int64_t>(blockIdx.x) * kWalkWarps + (threadIdx.x >> 5);
@@ -100,14 +103,16 @@ __global__ void __launch_bounds__(kWalkThreads, 1) walk(const WalkParams p) {
     for (int ti = 0; ti < ntiles; ++ti) {
         const int t_q0 = full ? 0 : p.q_begin + ti * cap_rows;          // first staged row
         const int t_rows = full ? p.Q : min(cap_rows, p.q_end - t_q0);  // staged rows
+        const int t_s0 = t_q0 & ~3;                                     // first row in the tile
         const int w_q0 = full ? p.q_begin : t_q0;                       // first start state
         const int w_rows = full ? nrows : t_rows;
         if (!raw) {
             if (ti > 0) __syncthreads();  // every warp is done with the previous tile
             if (threadIdx.x == 0) {
-                const uint32_t bytes = static_cast<uint32_t>(t_rows) * row_bytes;
+                const uint32_t bytes =
+                    (static_cast<uint32_t>(t_q0 - t_s0 + t_rows) * row_bytes + 15u) / 16u * 16u;
                 const uint8_t* src =
-                    reinterpret_cast<const uint8_t*>(gtab) + static_cast<size_t>(t_q0) * row_bytes;
+                    reinterpret_cast<const uint8_t*>(gtab) + static_cast<size_t>(t_s0) * row_bytes;
                 mbar_expect_tx(&bar, bytes);
                 for (uint32_t o = 0; o < bytes; o += kBulkChunk)
                     bulk_copy_g2s(smem_raw + o, src + o, min(kBulkChunk, bytes - o), &bar);
@@ -130,7 +135,7 @@ __global__ void __launch_bounds__(kWalkThreads, 1) walk(const WalkParams p) {
             if (raw) {
                 walk_task_raw<OutT, HAS_OUT>(p, q0, nq, g, lane);
             } else {
-                const TabT* first = tile + static_cast<size_t>(q0 - t_q0) * Cs;
+                const TabT* first = tile + static_cast<size_t>(q0 - t_s0) * Cs;
                 const bool has_eos = (p.eos_id >= 0) && ((p.eos_id >> 5) == g);
                 if (has_eos) {  // rare: one group in the whole vocabulary
                     if (full)

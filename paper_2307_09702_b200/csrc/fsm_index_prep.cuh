@@ -157,7 +157,7 @@ prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab
         raw_first = token_raw(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id,
                               static_cast<int64_t>(blockIdx.x) * kPrepTokens + tid, &bad_tok);
     const int C = derive_classes(partial, nparts, cs, s_cls, s_rep);
-    const int Cs = (C + 1 + 7) & ~7;
+    const int Cs = table_row_stride<TabT>(C);
     const bool two = C <= kTwoLevelMaxC;
     if (blockIdx.x == 0) {
         if (tid < 256) cls_out[tid] = s_cls[tid];

@@ -429,7 +429,8 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
     const int C = p.meta->C;
     const uint32_t Cs = p.meta->Cs;
     const bool two_level = p.meta->two_level != 0;
-    const uint64_t table_bytes = static_cast<uint64_t>(p.Q) * Cs * sizeof(TabT);
+    // (a bulk copy moves multiples of 16 bytes; the table's workspace has the slack)
+    const uint64_t table_bytes = (static_cast<uint64_t>(p.Q) * Cs * sizeof(TabT) + 15) / 16 * 16;
     const bool full = table_bytes <= table_cap;
     for (int i = threadIdx.x; i < 257; i += kWalkThreads) s_gstart[i] = p.gstart[i];
     if (full) {
