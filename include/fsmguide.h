@@ -134,10 +134,10 @@ int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* accept,
  * exits.  The call allocates and frees nothing.
  *
  *   - Size limit: the array holds the compressed transition table and the class
- *     records of the tokens; it has no room for the survivor lists of the faster
- *     work-avoiding walk, so this entry point always uses the dense walk (same
+ *     records of the tokens; it has no room for the scratch of the faster
+ *     work-avoiding walks, so this entry point always uses the dense walk (same
  *     results, lower throughput).  The build is refused with FSM_ERR_WORKSPACE,
- *     before anything is enqueued, when that scratch (about 330 KB + 528 bytes per
+ *     before anything is enqueued, when that scratch (about 270 KB + 528 bytes per
  *     state + 20 bytes per token) exceeds FSM_STATIC_SCRATCH_BYTES - as a guide: about
  *     1,000 states with 55,000 tokens, or 2,000 states with 30,000 tokens.  Larger
  *     problems need fsm_index_build and a workspace.
