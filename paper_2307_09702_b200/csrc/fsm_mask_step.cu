@@ -171,12 +171,19 @@ __device__ __forceinline__ float gumbel_score(float x, uint32_t v, uint32_t row,
     return __fmaf_rn(x, p.inv_temperature, -ln_rn(y));
 }
 
-// Masks one vector of NW words in place and folds the scores of its allowed entries into
-// the thread's best (score, id).  Ids only grow within a thread, so a strict comparison
-// keeps the lowest id among equal scores.
+// The better candidate has the larger score, or an equal score and the lower id (whatever
+// the visiting order).
+__device__ __forceinline__ void take_better(Best& a, float score, int id) {
+    if (a.idx == kNone || score > a.val || (score == a.val && id < a.idx)) {
+        a.val = score;
+        a.idx = id;
+    }
+}
+
+// Scores the allowed entries of one vector on the spot (rows that are not 32-byte aligned).
 template <typename T, int NW>
-__device__ __forceinline__ void process_sample(uint32_t (&w)[NW], uint32_t bits, int first_id,
-                                               uint32_t row, const StepParams& p, Best& best) {
+__device__ __forceinline__ void score_vector(const uint32_t (&w)[NW], uint32_t bits, int first_id,
+                                             uint32_t row, const StepParams& p, Best& best) {
     constexpr int PW = Elem<T>::kPerWord;
     uint32_t todo = bits;
     while (todo) {
@@ -185,14 +192,77 @@ __device__ __forceinline__ void process_sample(uint32_t (&w)[NW], uint32_t bits,
         uint32_t word = w[0];
 #pragma unroll
         for (int i = 1; i < NW; ++i) word = (j / PW == i) ? w[i] : word;
-        const float score = gumbel_score(Elem<T>::get(word, j % PW), first_id + j, row, p);
-        if (best.idx == kNone || score > best.val) {
-            best.val = score;
-            best.idx = first_id + j;
-        }
+        take_better(best, gumbel_score(Elem<T>::get(word, j % PW), first_id + j, row, p), first_id + j);
     }
+}
+
+template <typename T, int NW>
+__device__ __forceinline__ void mask_vector(uint32_t (&w)[NW], uint32_t bits) {
+    constexpr int PW = Elem<T>::kPerWord;
 #pragma unroll
     for (int i = 0; i < NW; ++i) w[i] = Elem<T>::select(w[i], (bits >> (i * PW)) & ((1u << PW) - 1u));
+}
+
+// Pool of allowed entries of one warp.  Few entries of a vector are allowed (one in
+// eighteen in the benchmark's index), so scoring them lane by lane would run the draw with
+// most lanes idle; instead every lane appends its (logit, id) pairs to the warp's queue and
+// the warp scores 32 queued entries at a time.  kQueue holds the leftovers of one round
+// (< 32) plus every entry of one 32-byte vector per lane (at most 16 bf16 values).
+constexpr int kQueue = 32 + 16 * 32;
+struct WarpQueue {
+    float x[kQueue];
+    int id[kQueue];
+};
+
+// All 32 lanes call this with their vector (bits == 0: nothing to add).
+template <typename T, int NW>
+__device__ __forceinline__ void pool_vector(const uint32_t (&w)[NW], uint32_t bits, int first_id,
+                                            uint32_t row, const StepParams& p, WarpQueue& q, int& qn,
+                                            Best& best) {
+    constexpr int PW = Elem<T>::kPerWord;
+    const int lane = threadIdx.x & 31;
+    const int mine = __popc(bits);
+    int incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int o = __shfl_up_sync(kFullWarp, incl, off);
+        if (lane >= off) incl += o;
+    }
+    const int total = __shfl_sync(kFullWarp, incl, 31);
+    if (total == 0) return;
+    int at = qn + incl - mine;
+    uint32_t todo = bits;
+    while (todo) {
+        const int j = __ffs(todo) - 1;
+        todo &= todo - 1;
+        uint32_t word = w[0];
+#pragma unroll
+        for (int i = 1; i < NW; ++i) word = (j / PW == i) ? w[i] : word;
+        q.x[at] = Elem<T>::get(word, j % PW);
+        q.id[at] = first_id + j;
+        ++at;
+    }
+    qn += total;
+    __syncwarp();
+    int head = 0;
+    for (; qn - head >= 32; head += 32)
+        take_better(best, gumbel_score(q.x[head + lane], q.id[head + lane], row, p), q.id[head + lane]);
+    if (head > 0) {  // leftovers to the front
+        const int rem = qn - head;
+        float x = 0.0f;
+        int id = 0;
+        if (lane < rem) {
+            x = q.x[head + lane];
+            id = q.id[head + lane];
+        }
+        __syncwarp();
+        if (lane < rem) {
+            q.x[lane] = x;
+            q.id[lane] = id;
+        }
+        qn = rem;
+    }
+    __syncwarp();
 }
 
 template <typename T, bool WRITE, bool SAMPLE>
@@ -200,6 +270,7 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
     cg::cluster_group cluster = cg::this_cluster();
     __shared__ Best warp_best[kStepWarps];
     __shared__ Best cta_best[8];  // slot r of the cluster's first CTA receives CTA r's result
+    __shared__ WarpQueue queues[SAMPLE ? kStepWarps : 1];
 
     const int k = p.k;
     const int row = blockIdx.x / k;
@@ -234,7 +305,11 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
         constexpr int kUnroll = 4, kGroup = 8;
         const int nvec = p.N / EPV;
         constexpr uint32_t kBitsMask = (EPV == 32) ? 0xFFFFFFFFu : ((1u << EPV) - 1u);
-        for (int g0 = tid; g0 < nvec; g0 += nthreads * kGroup) {
+        WarpQueue& queue = queues[SAMPLE ? (threadIdx.x >> 5) : 0];
+        int qn = 0;
+        // (the bound is the same for the 32 lanes of a warp: the pooled draw is a warp-wide step)
+        for (int g0 = tid; g0 - (SAMPLE ? static_cast<int>(threadIdx.x & 31) : 0) < nvec;
+             g0 += nthreads * kGroup) {
             uint32_t bits[kGroup];
 #pragma unroll
             for (int u = 0; u < kGroup; ++u) {
@@ -252,10 +327,11 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
                     const int vi = g0 + (h + u) * nthreads;
+                    if (SAMPLE) pool_vector<T, 8>(v[u].w, bits[h + u], vi * EPV, row, p, queue, qn, best);
                     if (vi < nvec) {
                         if (bits[h + u] != 0) {
                             if (SAMPLE)
-                                process_sample<T, 8>(v[u].w, bits[h + u], vi * EPV, row, p, best);
+                                mask_vector<T, 8>(v[u].w, bits[h + u]);
                             else
                                 process<T, 8>(v[u].w, bits[h + u], vi, tb);
                         } else {
@@ -267,6 +343,9 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
                 }
             }
         }
+        if (SAMPLE && static_cast<int>(threadIdx.x & 31) < qn)  // what is left in the pool
+            take_better(best, gumbel_score(queue.x[threadIdx.x & 31], queue.id[threadIdx.x & 31], row, p),
+                        queue.id[threadIdx.x & 31]);
         done = nvec * EPV;
     } else {
         const int nvec = p.N / EPH;
@@ -277,10 +356,12 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
             if (bits != 0) {
                 const uint4 v = *reinterpret_cast<const uint4*>(in + e0);
                 w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
-                if (SAMPLE)
-                    process_sample<T, 4>(w, bits, e0, row, p, best);
-                else
+                if (SAMPLE) {
+                    score_vector<T, 4>(w, bits, e0, row, p, best);
+                    mask_vector<T, 4>(w, bits);
+                } else {
                     process<T, 4>(w, bits, vi, tb);
+                }
             } else {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) w[i] = Elem<T>::kNegInfWord;
@@ -313,8 +394,9 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
             if (allowed) {
                 float x = sizeof(T) == 4 ? __uint_as_float(static_cast<uint32_t>(raw))
                                          : __uint_as_float(static_cast<uint32_t>(raw) << 16);
-                if (SAMPLE) x = gumbel_score(x, e, row, p);
-                if (best.idx == kNone || x > best.val) {  // tail ids exceed every vector id
+                if (SAMPLE) {
+                    take_better(best, gumbel_score(x, e, row, p), e);
+                } else if (best.idx == kNone || x > best.val) {  // tail ids exceed every vector id
                     best.val = x;
                     best.idx = e;
                 }
