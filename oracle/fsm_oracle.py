@@ -162,3 +162,25 @@ def ln_f32(x: float) -> float:
 
 def gumbel_f32(bits: int) -> float:
     return float(_load().oracle_gumbel_f32(bits & 0xFFFFFFFF))
+
+
+def index_csr(trans, accept, vocab_bytes, vocab_offsets, dead_state, eos_id=-1, threads=1):
+    """The index in the paper's own form - sigma: state -> set of allowed tokens - as
+    compressed rows: ``(allowed_mask, row_offsets int64 [Q+1], tokens int32 [nnz],
+    next int32 [nnz])`` with row q's allowed tokens in increasing id order at
+    ``row_offsets[q] .. row_offsets[q+1]-1`` and the state each one leads to beside it.
+    Written out from the dense definition: an entry for every set bit, nothing else."""
+    mask, nxt, _ = index_build(trans, accept, vocab_bytes, vocab_offsets, dead_state, eos_id,
+                               threads=threads)
+    Q, N = nxt.shape
+    offsets = np.zeros(Q + 1, dtype=np.int64)
+    toks, nexts = [], []
+    for q in range(Q):
+        bits = np.unpackbits(mask[q].view(np.uint8), bitorder="little")[:N]
+        ids = np.flatnonzero(bits).astype(np.int32)
+        toks.append(ids)
+        nexts.append(nxt[q, ids])
+        offsets[q + 1] = offsets[q] + len(ids)
+    tokens = np.concatenate(toks) if toks else np.zeros(0, np.int32)
+    nexts = np.concatenate(nexts).astype(np.int32) if nexts else np.zeros(0, np.int32)
+    return mask, offsets, tokens, nexts
