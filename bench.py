@@ -349,6 +349,34 @@ def run_ours(args):
     u16_ms = time_build(fg.FSM_STATE_U16, True)
     maskonly_ms = time_build(fg.FSM_STATE_I32, False)
 
+    def time_csr(n=20):
+        """The index as compressed rows (allowed token lists with end states)."""
+        cap = int(0.08 * w.Q * w.N)
+        off = torch.empty(w.Q + 1, dtype=torch.int64, device=dev)
+        ctok = torch.empty(cap, dtype=torch.int32, device=dev)
+        cnext = torch.empty(cap, dtype=torch.int32, device=dev)
+
+        def run():
+            rc = fg.fsm_index_build_csr(idx.trans, idx.accept, idx.vocab_bytes, idx.vocab_offsets,
+                                        idx.vocab_nbytes, w.Q, w.N, d.dead, w.eos_id, idx.allowed_mask,
+                                        off, ctok, cnext, cap, idx.workspace, idx.workspace_bytes,
+                                        idx.status)
+            assert rc == 0
+        for _ in range(3):
+            run()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(n):
+            run()
+        b.record()
+        torch.cuda.synchronize()
+        assert int(idx.status.item()) == 0, "compressed-row capacity too small"
+        return a.elapsed_time(b) / n, int(off[-1].item())
+
+    csr_ms, csr_nnz = time_csr()
+    idx.build()    # the dense index again, for the end-to-end loop below
+
     # ---- end to end: host buffers in, host results out, through the same calls
     host = {k: torch.from_numpy(np.ascontiguousarray(v)).pin_memory() for k, v in {
         "trans": d.trans, "accept": d.accept, "vb": w.vocab_bytes, "vo": w.vocab_offsets,
@@ -396,8 +424,8 @@ def run_ours(args):
         return float(t.item())
 
     (total_ms, build_ms, mask_ms, mask_in_step_ms, walk_ms_mean, e2e_s, u16_ms, maskonly_ms,
-     sample_ms) = map(allmax, (total_ms, build_ms, mask_ms, mask_in_step_ms, walk_ms_mean, e2e_s,
-                               u16_ms, maskonly_ms, sample_ms))
+     sample_ms, csr_ms) = map(allmax, (total_ms, build_ms, mask_ms, mask_in_step_ms, walk_ms_mean,
+                                       e2e_s, u16_ms, maskonly_ms, sample_ms, csr_ms))
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -450,6 +478,11 @@ def run_ours(args):
                              "smem_lookup_bound_frac": (walks / (maskonly_ms * 1e-3)) / SMEM_LOOKUP_BOUND,
                              "note": "bound = 148 SMs x 32 lookups/clk x 1.965 GHz / 1.157 lookups "
                                      "per walk (oracle-counted) = 8.04e12 walks/s"},
+            "compressed_rows": {"us": csr_ms * 1e3, "walks_per_s": walks / (csr_ms * 1e-3),
+                                "entries": csr_nnz,
+                                "output_bytes": csr_nnz * 8 + (w.Q + 1) * 8 + w.Q * w.W * 4,
+                                "note": "fsm_index_build_csr: bitmask + per-state token lists with "
+                                        "end states instead of the dense table"},
             "note": "whole builds (all launches), per-rank"},
         "clocks": clocks,
         "e2e": {"value": walks * world / e2e_s, "unit": UNIT, "ms_per_step": e2e_s * 1e3,

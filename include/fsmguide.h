@@ -45,6 +45,8 @@ extern "C" {
 #define FSM_FLAG_CLASS_SPLIT 8   /* informational: two byte columns hashed alike but differ;
                                     the build took the uncompressed path (still exact) */
 #define FSM_FLAG_WAIT_TIMEOUT 16 /* a bounded wait on an on-chip copy gave up; output invalid */
+#define FSM_FLAG_CSR_OVERFLOW 32 /* fsm_index_build_csr: more allowed pairs than `capacity`;
+                                    row_offsets is complete, entries beyond capacity are missing */
 
 typedef enum { FSM_STATE_I32 = 0, FSM_STATE_U16 = 1 } fsm_state_dtype;
 typedef enum { FSM_LOGITS_F32 = 0, FSM_LOGITS_BF16 = 1 } fsm_logits_dtype;
@@ -118,6 +120,32 @@ int fsm_index_build_rows(const int32_t* dfa_trans, const uint8_t* accept,
                          uint32_t* allowed_mask, void* next_state, int32_t state_dtype,
                          void* workspace, size_t workspace_bytes, int32_t* status_word,
                          void* cuda_stream);
+
+/*
+ * The index in the paper's own form (Section 3, Algorithm 4: sigma maps a state to the
+ * *set* of allowed tokens), as compressed rows.  Most (state, token) pairs are not
+ * allowed (the paper notes that the map's memory grows with the number of states only),
+ * so this form is a small fraction of the dense next-state table.
+ *
+ *   allowed_mask   out, as fsm_index_build.
+ *   row_offsets    out, int64 [Q+1], 8-byte aligned: row q's entries are
+ *                  row_offsets[q] .. row_offsets[q+1]-1; row_offsets[Q] is the number of
+ *                  allowed pairs.
+ *   csr_tokens     out, int32 [capacity]: the allowed token ids of each row, increasing.
+ *   csr_next       out, int32 [capacity]: the state each of them leads to (for EOS: the
+ *                  state itself).
+ *   capacity       entries the two arrays hold.  If the index has more, the first
+ *                  `capacity` entries are written, FSM_FLAG_CSR_OVERFLOW is raised and
+ *                  row_offsets (always complete) tells the size needed.
+ * Other arguments, workspace and status word as fsm_index_build.
+ */
+int fsm_index_build_csr(const int32_t* dfa_trans, const uint8_t* accept,
+                        const uint8_t* vocab_bytes, const int32_t* vocab_offsets,
+                        int64_t vocab_nbytes, int32_t Q, int32_t N, int32_t dead_state,
+                        int32_t eos_id, uint32_t* allowed_mask, int64_t* row_offsets,
+                        int32_t* csr_tokens, int32_t* csr_next, int64_t capacity,
+                        void* workspace, size_t workspace_bytes, int32_t* status_word,
+                        void* cuda_stream);
 
 /*
  * Index build without caller-provided scratch.  The paper has no counterpart:
@@ -224,6 +252,22 @@ int guided_sample_step(const void* logits_in, void* logits_out, int32_t logits_d
                        const void* next_state, int32_t state_dtype, int32_t Q, int32_t N,
                        int32_t B, int32_t dead_state, int32_t eos_id, float inv_temperature,
                        uint64_t seed, uint64_t draw, int32_t* status_word, void* cuda_stream);
+
+/*
+ * The decode step on the compressed-row index of fsm_index_build_csr: guided_mask_step
+ * (sample == 0) or guided_sample_step (sample != 0; inv_temperature, seed and draw as
+ * there), except that the next state of the chosen token is found by binary search among
+ * the row's tokens instead of in a dense table.  Same masking, selection and bookkeeping,
+ * same results.  A chosen token whose entry is missing (index built with too small a
+ * capacity, FSM_FLAG_CSR_OVERFLOW) sends the row to the dead state.
+ */
+int guided_step_csr(const void* logits_in, void* logits_out, int32_t logits_dtype,
+                    int64_t row_stride, int32_t* states, uint8_t* finished, int32_t* tokens_out,
+                    const uint32_t* allowed_mask, const int64_t* row_offsets,
+                    const int32_t* csr_tokens, const int32_t* csr_next, int32_t Q, int32_t N,
+                    int32_t B, int32_t dead_state, int32_t eos_id, int32_t sample,
+                    float inv_temperature, uint64_t seed, uint64_t draw, int32_t* status_word,
+                    void* cuda_stream);
 
 /*
  * Tuning and test hooks (no counterpart in the paper).  Sets a process-wide knob

@@ -8,12 +8,12 @@ built library raises.
 from .batching import stack_automata
 from .binding import (FSM_LOGITS_BF16, FSM_LOGITS_F32, FSM_STATE_I32, FSM_STATE_U16, FsmError,
                       GuidedIndex, fsm_debug_set, fsm_device_check, fsm_index_build,
-                      fsm_index_build_rows, fsm_index_build_static, fsm_index_workspace_bytes, fsm_profile_read, fsm_status_string,
-                      guided_mask_step, guided_sample_step, lib, library_path)
+                      fsm_index_build_csr, fsm_index_build_rows, fsm_index_build_static, fsm_index_workspace_bytes, fsm_profile_read, fsm_status_string,
+                      guided_mask_step, guided_sample_step, guided_step_csr, lib, library_path)
 
 __all__ = [
     "FSM_LOGITS_BF16", "FSM_LOGITS_F32", "FSM_STATE_I32", "FSM_STATE_U16", "FsmError",
     "GuidedIndex", "fsm_debug_set", "fsm_device_check", "fsm_index_build",
-    "fsm_index_build_rows", "fsm_index_build_static", "fsm_index_workspace_bytes", "fsm_profile_read", "fsm_status_string",
-    "guided_mask_step", "guided_sample_step", "lib", "library_path", "stack_automata",
+    "fsm_index_build_csr", "fsm_index_build_rows", "fsm_index_build_static", "fsm_index_workspace_bytes", "fsm_profile_read", "fsm_status_string",
+    "guided_mask_step", "guided_sample_step", "guided_step_csr", "lib", "library_path", "stack_automata",
 ]

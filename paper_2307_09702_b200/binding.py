@@ -69,6 +69,12 @@ def lib() -> ctypes.CDLL:
         L.guided_sample_step.argtypes = [vp, vp, i32, i64, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32,
                                          i32, ctypes.c_float, ctypes.c_uint64, ctypes.c_uint64, vp, vp]
         L.guided_sample_step.restype = ctypes.c_int
+        L.fsm_index_build_csr.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, vp, vp, i64,
+                                          vp, sz, vp, vp]
+        L.fsm_index_build_csr.restype = ctypes.c_int
+        L.guided_step_csr.argtypes = [vp, vp, i32, i64, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32,
+                                      i32, i32, ctypes.c_float, ctypes.c_uint64, ctypes.c_uint64, vp, vp]
+        L.guided_step_csr.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -161,6 +167,27 @@ def guided_sample_step(logits_in, logits_out, logits_dtype, row_stride, states, 
                                     dead_state, eos_id, inv_temperature,
                                     seed & 0xFFFFFFFFFFFFFFFF, draw & 0xFFFFFFFFFFFFFFFF,
                                     _ptr(status_word), _stream(stream))
+
+
+def fsm_index_build_csr(dfa_trans, accept, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state,
+                        eos_id, allowed_mask, row_offsets, csr_tokens, csr_next, capacity, workspace,
+                        workspace_bytes, status_word=None, stream=None) -> int:
+    return lib().fsm_index_build_csr(_ptr(dfa_trans), _ptr(accept), _ptr(vocab_bytes),
+                                     _ptr(vocab_offsets), vocab_nbytes, Q, N, dead_state, eos_id,
+                                     _ptr(allowed_mask), _ptr(row_offsets), _ptr(csr_tokens),
+                                     _ptr(csr_next), capacity, _ptr(workspace), workspace_bytes,
+                                     _ptr(status_word), _stream(stream))
+
+
+def guided_step_csr(logits_in, logits_out, logits_dtype, row_stride, states, finished, tokens_out,
+                    allowed_mask, row_offsets, csr_tokens, csr_next, Q, N, B, dead_state, eos_id,
+                    sample=0, inv_temperature=1.0, seed=0, draw=0, status_word=None, stream=None) -> int:
+    return lib().guided_step_csr(_ptr(logits_in), _ptr(logits_out), logits_dtype, row_stride,
+                                 _ptr(states), _ptr(finished), _ptr(tokens_out), _ptr(allowed_mask),
+                                 _ptr(row_offsets), _ptr(csr_tokens), _ptr(csr_next), Q, N, B,
+                                 dead_state, eos_id, sample, inv_temperature,
+                                 seed & 0xFFFFFFFFFFFFFFFF, draw & 0xFFFFFFFFFFFFFFFF,
+                                 _ptr(status_word), _stream(stream))
 
 
 class GuidedIndex:

@@ -18,6 +18,7 @@
 #include "fsm_index_prep.cuh"
 #include "fsm_index_sparse.cuh"
 #include "fsm_index_bucket.cuh"
+#include "fsm_index_csr.cuh"
 
 extern "C" size_t fsm_index_workspace_bytes(int32_t Q, int32_t N, int64_t vocab_nbytes) {
     if (Q <= 0 || N <= 0 || vocab_nbytes < 0) return 0;
@@ -100,7 +101,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
                               vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
                               ws.partial, hash_blocks, ws.meta, ws.cls, static_cast<int32_t*>(ws.table),
                               tok_cls, ws.tok_len, live, ws.gcount, count2, planes,
-                              status_word) != cudaSuccess)
+                              bucket ? ws.tok_head : nullptr, status_word) != cudaSuccess)
             return FSM_ERR_CUDA;
     } else {
         auto k = prepare_all<uint16_t>;
@@ -111,7 +112,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
                               vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
                               ws.partial, hash_blocks, ws.meta, ws.cls, static_cast<uint16_t*>(ws.table),
                               tok_cls, ws.tok_len, live, ws.gcount, count2, planes,
-                              status_word) != cudaSuccess)
+                              bucket ? ws.tok_head : nullptr, status_word) != cudaSuccess)
             return FSM_ERR_CUDA;
     }
     if (sparse) {
@@ -262,4 +263,51 @@ extern "C" int fsm_index_build_static(const int32_t* dfa_trans, const uint8_t* a
     return build_rows_impl(dfa_trans, accept, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N,
                            dead_state, eos_id, 0, Q, allowed_mask, next_state, state_dtype, scratch,
                            FSM_STATIC_SCRATCH_BYTES, status_word, cuda_stream, true);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Compressed rows: a bitmask-only build, then the rows are cut out of the bitmask.
+extern "C" int fsm_index_build_csr(const int32_t* dfa_trans, const uint8_t* accept,
+                                   const uint8_t* vocab_bytes, const int32_t* vocab_offsets,
+                                   int64_t vocab_nbytes, int32_t Q, int32_t N, int32_t dead_state,
+                                   int32_t eos_id, uint32_t* allowed_mask, int64_t* row_offsets,
+                                   int32_t* csr_tokens, int32_t* csr_next, int64_t capacity,
+                                   void* workspace, size_t workspace_bytes, int32_t* status_word,
+                                   void* cuda_stream) {
+    using namespace fsm;
+    if (!row_offsets || (capacity > 0 && (!csr_tokens || !csr_next))) return FSM_ERR_NULL;
+    if (capacity < 0) return FSM_ERR_SHAPE;
+    auto misaligned = [](const void* p, size_t a) { return reinterpret_cast<uintptr_t>(p) % a != 0; };
+    if (misaligned(row_offsets, 8) || misaligned(csr_tokens, 4) || misaligned(csr_next, 4))
+        return FSM_ERR_ALIGN;
+    const int rc = build_rows_impl(dfa_trans, accept, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N,
+                                   dead_state, eos_id, 0, Q, allowed_mask, nullptr, FSM_STATE_I32,
+                                   workspace, workspace_bytes, status_word, cuda_stream, false);
+    if (rc != FSM_OK) return rc;
+    const DeviceInfo& dev = device_info();
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    Workspace ws = carve(workspace, Q, N);
+    WalkParams p = {};
+    p.trans = dfa_trans;
+    p.accept = accept;
+    p.vocab_bytes = vocab_bytes;
+    p.vocab_offsets = vocab_offsets;
+    p.vocab_nbytes = vocab_nbytes;
+    p.Q = Q;
+    p.N = N;
+    p.G = (N + 31) / 32;
+    p.dead = dead_state;
+    p.eos_id = eos_id;
+    p.q_begin = 0;
+    p.q_end = Q;
+    p.mask = allowed_mask;
+    p.status = status_word;
+    const int blocks = Q < 8 * dev.sm_count ? Q : 8 * dev.sm_count;
+    csr_count<<<blocks, kCsrThreads, 0, stream>>>(allowed_mask, p.G, Q, ws.row_count);
+    csr_scan<<<1, 1024, 0, stream>>>(ws.row_count, Q, row_offsets, capacity, status_word);
+    const int fill_blocks = Q < 16 * dev.sm_count ? Q : 16 * dev.sm_count;
+    const int fill_parts = p.G >= 4 * 32 * kFillWarps ? 4 : 1;
+    csr_fill<<<dim3(fill_blocks, fill_parts), kFillThreads, 0, stream>>>(p, ws.tok_head, row_offsets, csr_tokens, csr_next,
+                                                       capacity);
+    return cudaGetLastError() == cudaSuccess ? FSM_OK : FSM_ERR_CUDA;
 }

@@ -46,6 +46,8 @@ struct Workspace {
     // bucket walk: bit planes of the one-byte tokens by class, live classes of every state
     uint32_t* planes;    // [256][W] bit v of plane c: token v is the one byte of class c
     uint32_t* live;      // [Q][8] bit c: state reads class c
+    int32_t* row_count;  // [Q] allowed tokens per row (compressed-row build)
+    uint16_t* tok_head;  // [N] first byte | min(length, 255) << 8 of every token
     size_t bytes;        // everything above
     size_t dense_bytes;  // the part in front of `survivors`: enough for the dense walk
 };
@@ -95,6 +97,8 @@ inline Workspace carve(void* base, int32_t Q, int32_t N) {
     w.survivors = take(ctas * slice_slots * (Q <= 65535 ? 4 : 8));
     w.planes = reinterpret_cast<uint32_t*>(take(256 * (G32 / 32) * sizeof(uint32_t)));
     w.live = reinterpret_cast<uint32_t*>(take(static_cast<size_t>(Q) * 8 * sizeof(uint32_t)));
+    w.row_count = reinterpret_cast<int32_t*>(take(static_cast<size_t>(Q) * sizeof(int32_t)));
+    w.tok_head = reinterpret_cast<uint16_t*>(take(static_cast<size_t>(N) * sizeof(uint16_t)));
     w.bytes = off;
     return w;
 }

@@ -139,7 +139,8 @@ prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab
             IndexMeta* meta, uint8_t* __restrict__ cls_out, TabT* __restrict__ table,
             uint4* __restrict__ tok_cls, uint8_t* __restrict__ tok_len,
             uint32_t* __restrict__ live, int32_t* __restrict__ gcount,
-            int32_t* __restrict__ count2, uint32_t* __restrict__ planes, int32_t* status) {
+            int32_t* __restrict__ count2, uint32_t* __restrict__ planes,
+            uint16_t* __restrict__ tok_head, int32_t* status) {
     extern __shared__ int s_cnt[];  // [kKeys] when keys are counted
     __shared__ ClassScratch cs;
     __shared__ uint8_t s_cls[256], s_rep[256];
@@ -252,6 +253,8 @@ prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab
                                      ? raw_first
                                      : token_raw(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, v, &bad);
             const TokenInfo t = token_classify(raw, s_cls);
+            if (tok_head != nullptr && v < N)  // first byte and length, for the compressed rows
+                tok_head[v] = static_cast<uint16_t>(raw.b0 | (static_cast<uint32_t>(raw.len) << 8));
             if (t.len > 0) {
                 atomicAdd(&hist[t.first], 1);
                 atomicAdd(&s_cnt[bucket_key(two, t.first, t.second_key)], 1);

@@ -34,6 +34,10 @@ struct StepParams {
     int32_t state_u16;
     int32_t Q, N, W, B, dead, eos_id, k;
     int32_t* status;
+    // compressed-row index (csr_offsets != nullptr): next states by search in the row
+    const int64_t* csr_offsets;
+    const int32_t* csr_tokens;
+    const int32_t* csr_next;
     // sampling
     float inv_temperature;
     uint32_t seed_lo, seed_hi, draw_lo, draw_hi;
@@ -214,6 +218,17 @@ struct WarpQueue {
     int id[kQueue];
 };
 
+// The queues of a CTA; the greedy variant has none.
+template <bool SAMPLE> struct QueueStore {
+    __device__ static WarpQueue* get() {
+        __shared__ WarpQueue queues[kStepWarps];
+        return queues;
+    }
+};
+template <> struct QueueStore<false> {
+    __device__ static WarpQueue* get() { return nullptr; }
+};
+
 // All 32 lanes call this with their vector (bits == 0: nothing to add).
 template <typename T, int NW>
 __device__ __forceinline__ void pool_vector(const uint32_t (&w)[NW], uint32_t bits, int first_id,
@@ -270,7 +285,6 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
     cg::cluster_group cluster = cg::this_cluster();
     __shared__ Best warp_best[kStepWarps];
     __shared__ Best cta_best[8];  // slot r of the cluster's first CTA receives CTA r's result
-    __shared__ WarpQueue queues[SAMPLE ? kStepWarps : 1];
 
     const int k = p.k;
     const int row = blockIdx.x / k;
@@ -305,7 +319,7 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
         constexpr int kUnroll = 4, kGroup = 8;
         const int nvec = p.N / EPV;
         constexpr uint32_t kBitsMask = (EPV == 32) ? 0xFFFFFFFFu : ((1u << EPV) - 1u);
-        WarpQueue& queue = queues[SAMPLE ? (threadIdx.x >> 5) : 0];
+        WarpQueue& queue = QueueStore<SAMPLE>::get()[SAMPLE ? (threadIdx.x >> 5) : 0];
         int qn = 0;
         // (the bound is the same for the 32 lanes of a warp: the pooled draw is a warp-wide step)
         for (int g0 = tid; g0 - (SAMPLE ? static_cast<int>(threadIdx.x & 31) : 0) < nvec;
@@ -438,9 +452,24 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
             p.tokens[row] = b.idx;
         } else {
             p.tokens[row] = b.idx;
-            const size_t at = static_cast<size_t>(q) * p.N + b.idx;
-            p.states[row] = p.state_u16 ? static_cast<int32_t>(static_cast<const uint16_t*>(p.next)[at])
-                                        : static_cast<const int32_t*>(p.next)[at];
+            if (p.csr_offsets != nullptr) {
+                // the row's tokens are in increasing order: binary search for the chosen one
+                int64_t lo = p.csr_offsets[q], hi = p.csr_offsets[q + 1];
+                while (lo < hi) {
+                    const int64_t mid = (lo + hi) >> 1;
+                    if (p.csr_tokens[mid] < b.idx)
+                        lo = mid + 1;
+                    else
+                        hi = mid;
+                }
+                const bool found = lo < p.csr_offsets[q + 1] && p.csr_tokens[lo] == b.idx;
+                p.states[row] = found ? p.csr_next[lo] : p.dead;  // (an entry lost to a too small
+                                                                  // capacity leads to dead)
+            } else {
+                const size_t at = static_cast<size_t>(q) * p.N + b.idx;
+                p.states[row] = p.state_u16 ? static_cast<int32_t>(static_cast<const uint16_t*>(p.next)[at])
+                                            : static_cast<const int32_t*>(p.next)[at];
+            }
         }
     }
 }
@@ -471,11 +500,12 @@ int step_impl(const void* logits_in, void* logits_out, int32_t logits_dtype, int
               const uint32_t* allowed_mask, const void* next_state, int32_t state_dtype, int32_t Q,
               int32_t N, int32_t B, int32_t dead_state, int32_t eos_id, bool sample,
               float inv_temperature, uint64_t seed, uint64_t draw, int32_t* status_word,
-              void* cuda_stream) {
+              void* cuda_stream, const int64_t* csr_offsets = nullptr,
+              const int32_t* csr_tokens = nullptr, const int32_t* csr_next = nullptr) {
     using namespace fsm;
     if (Q <= 0 || N <= 0 || B < 0 || row_stride < N) return FSM_ERR_SHAPE;
-    if (!logits_in || !states || !finished || !tokens_out || !allowed_mask || !next_state)
-        return FSM_ERR_NULL;
+    if (!logits_in || !states || !finished || !tokens_out || !allowed_mask) return FSM_ERR_NULL;
+    if (csr_offsets ? (!csr_tokens || !csr_next) : !next_state) return FSM_ERR_NULL;
     if (logits_dtype != FSM_LOGITS_F32 && logits_dtype != FSM_LOGITS_BF16) return FSM_ERR_DTYPE;
     if (state_dtype != FSM_STATE_I32 && state_dtype != FSM_STATE_U16) return FSM_ERR_DTYPE;
     if (state_dtype == FSM_STATE_U16 && Q > 65535) return FSM_ERR_DTYPE;
@@ -524,6 +554,9 @@ int step_impl(const void* logits_in, void* logits_out, int32_t logits_dtype, int
     p.eos_id = eos_id;
     p.k = k;
     p.status = status_word;
+    p.csr_offsets = csr_offsets;
+    p.csr_tokens = csr_tokens;
+    p.csr_next = csr_next;
     p.inv_temperature = inv_temperature;
     p.seed_lo = static_cast<uint32_t>(seed);
     p.seed_hi = static_cast<uint32_t>(seed >> 32);
@@ -568,4 +601,23 @@ extern "C" int guided_sample_step(const void* logits_in, void* logits_out, int32
     return step_impl(logits_in, logits_out, logits_dtype, row_stride, states, finished, tokens_out,
                      allowed_mask, next_state, state_dtype, Q, N, B, dead_state, eos_id, true,
                      inv_temperature, seed, draw, status_word, cuda_stream);
+}
+
+extern "C" int guided_step_csr(const void* logits_in, void* logits_out, int32_t logits_dtype,
+                               int64_t row_stride, int32_t* states, uint8_t* finished,
+                               int32_t* tokens_out, const uint32_t* allowed_mask,
+                               const int64_t* row_offsets, const int32_t* csr_tokens,
+                               const int32_t* csr_next, int32_t Q, int32_t N, int32_t B,
+                               int32_t dead_state, int32_t eos_id, int32_t sample,
+                               float inv_temperature, uint64_t seed, uint64_t draw,
+                               int32_t* status_word, void* cuda_stream) {
+    if (!row_offsets) return FSM_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(row_offsets) % 8 != 0 ||
+        reinterpret_cast<uintptr_t>(csr_tokens) % 4 != 0 || reinterpret_cast<uintptr_t>(csr_next) % 4 != 0)
+        return FSM_ERR_ALIGN;
+    if (sample && (!(inv_temperature > 0.0f) || !(inv_temperature < 3.0e38f))) return FSM_ERR_RANGE;
+    return step_impl(logits_in, logits_out, logits_dtype, row_stride, states, finished, tokens_out,
+                     allowed_mask, nullptr, FSM_STATE_I32, Q, N, B, dead_state, eos_id, sample != 0,
+                     sample ? inv_temperature : 1.0f, seed, draw, status_word, cuda_stream,
+                     row_offsets, csr_tokens, csr_next);
 }
