@@ -77,7 +77,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
                         sparse_table_offset<int32_t>(N) + 4096 <= static_cast<size_t>(dev.smem_optin - 2048);
 
     const int hash_blocks = Q < kHashBlocks ? Q : kHashBlocks;
-    if (launch_on(hash_columns, dim3(hash_blocks), dim3(256 * kHashRowLanes), 0, stream,
+    if (launch_overlapped(hash_columns, dim3(hash_blocks), dim3(256 * kHashRowLanes), 0, stream,
                           dfa_trans, Q, dead_state, ws.partial, tune.weak_hash, ws.meta, ws.gcount,
                           ws.count2, ws.cursor2, ws.row_ctr, status_word) != cudaSuccess)
         return FSM_ERR_CUDA;
@@ -97,7 +97,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
         if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(kKeys * sizeof(int))) != cudaSuccess)
             return FSM_ERR_CUDA;
-        if (launch_on(k, dim3(prep_blocks), dim3(kPrepThreads), key_smem, stream, dfa_trans,
+        if (launch_overlapped(k, dim3(prep_blocks), dim3(kPrepThreads), key_smem, stream, dfa_trans,
                               vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
                               ws.partial, hash_blocks, ws.meta, ws.cls, static_cast<int32_t*>(ws.table),
                               tok_cls, ws.tok_len, live, ws.gcount, count2, planes,
@@ -108,7 +108,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
         if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(kKeys * sizeof(int))) != cudaSuccess)
             return FSM_ERR_CUDA;
-        if (launch_on(k, dim3(prep_blocks), dim3(kPrepThreads), key_smem, stream, dfa_trans,
+        if (launch_overlapped(k, dim3(prep_blocks), dim3(kPrepThreads), key_smem, stream, dfa_trans,
                               vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
                               ws.partial, hash_blocks, ws.meta, ws.cls, static_cast<uint16_t*>(ws.table),
                               tok_cls, ws.tok_len, live, ws.gcount, count2, planes,
@@ -120,7 +120,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
                                  static_cast<int>(sort_smem)) != cudaSuccess)
             return FSM_ERR_CUDA;
         const int sort_blocks = nchunks < dev.sm_count ? nchunks : dev.sm_count;
-        if (launch_on(sort_all, dim3(sort_blocks), dim3(kPrepThreads), sort_smem, stream,
+        if (launch_overlapped(sort_all, dim3(sort_blocks), dim3(kPrepThreads), sort_smem, stream,
                               vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, ws.meta, ws.cls,
                               ws.count2, ws.cursor2, ws.start2, ws.gstart, ws.srec,
                               ws.sid) != cudaSuccess)

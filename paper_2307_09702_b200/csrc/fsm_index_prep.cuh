@@ -26,6 +26,8 @@ hash_columns(const int32_t* __restrict__ trans, int32_t Q, int32_t dead,
              int32_t* __restrict__ cursor2, int32_t* __restrict__ row_ctr, int32_t* status) {
     __shared__ uint64_t part[kHashRowLanes][256];
     const int b = threadIdx.x & 255, rl = threadIdx.x >> 8;
+    pdl_launch_dependents();
+    // delta is an input of the build: it may be read while the previous kernel still runs
     uint64_t h = 0;
     bool bad = false;
 #pragma unroll 4
@@ -35,6 +37,7 @@ hash_columns(const int32_t* __restrict__ trans, int32_t Q, int32_t dead,
         bad |= static_cast<uint32_t>(v) >= static_cast<uint32_t>(Q);
         h += mix64((static_cast<uint64_t>(q) << 32) | static_cast<uint32_t>(v));
     }
+    pdl_wait();  // the workspace may still be in use by the kernels before this one
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         *row_ctr = 0;
         meta->any_bad = 0;
@@ -71,7 +74,7 @@ struct ClassScratch {
     uint32_t rep_bits[8];
 };
 
-__device__ __forceinline__ int derive_classes(const uint64_t* __restrict__ partial, int nparts,
+__device__ __forceinline__ int derive_classes(const uint64_t* partial, int nparts,
                                               ClassScratch& cs, uint8_t* s_cls, uint8_t* s_rep) {
     constexpr int kSlots = 1024;
     constexpr unsigned long long kEmpty = ~0ull;
@@ -135,7 +138,7 @@ template <typename TabT>
 __global__ void __launch_bounds__(kPrepThreads)
 prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab_bytes,
             const int32_t* __restrict__ vocab_offsets, int64_t vocab_nbytes, int32_t Q, int32_t N,
-            int32_t dead, int32_t eos_id, const uint64_t* __restrict__ partial, int nparts,
+            int32_t dead, int32_t eos_id, const uint64_t* partial, int nparts,
             IndexMeta* meta, uint8_t* __restrict__ cls_out, TabT* __restrict__ table,
             uint4* __restrict__ tok_cls, uint8_t* __restrict__ tok_len,
             uint32_t* __restrict__ live, int32_t* __restrict__ gcount,
@@ -157,6 +160,8 @@ prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab
     if (count2 != nullptr)
         raw_first = token_raw(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id,
                               static_cast<int64_t>(blockIdx.x) * kPrepTokens + tid, &bad_tok);
+    pdl_launch_dependents();
+    pdl_wait();  // the column hashes come from the kernel before
     const int C = derive_classes(partial, nparts, cs, s_cls, s_rep);
     const int Cs = table_row_stride<TabT>(C);
     const bool two = C <= kTwoLevelMaxC;
@@ -286,9 +291,8 @@ constexpr int kKeysPad = kScanPer * kPrepThreads;
 
 __global__ void __launch_bounds__(kPrepThreads)
 sort_all(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vocab_offsets,
-         int64_t vocab_nbytes, int32_t N, int32_t eos_id, const IndexMeta* __restrict__ meta,
-         const uint8_t* __restrict__ cls, const int32_t* __restrict__ count2,
-         int32_t* __restrict__ cursor2, int32_t* __restrict__ start2,
+         int64_t vocab_nbytes, int32_t N, int32_t eos_id, const IndexMeta* meta,
+         const uint8_t* cls, const int32_t* count2, int32_t* cursor2, int32_t* __restrict__ start2,
          int32_t* __restrict__ gstart, uint4* __restrict__ srec, int32_t* __restrict__ sid) {
     extern __shared__ int s_sort[];  // s_start[kKeysPad], s_cnt[kKeys]
     int* s_start = s_sort;
@@ -306,6 +310,8 @@ sort_all(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vo
         bytes_first[i] = i < raw_first.len ? vocab_bytes[raw_first.start + i] : 0;
     bytes_first[0] = static_cast<uint8_t>(raw_first.b0);
     bytes_first[1] = static_cast<uint8_t>(raw_first.b1);
+    pdl_launch_dependents();
+    pdl_wait();  // classes and key counts come from the kernel before
     if (tid < 256) s_cls[tid] = cls[tid];
     const bool two = meta->two_level != 0;
     const int nkeys = two ? kKeys : 256;
