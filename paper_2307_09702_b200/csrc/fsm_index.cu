@@ -78,7 +78,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
 
     const int hash_blocks = Q < kHashBlocks ? Q : kHashBlocks;
     if (launch_overlapped(hash_columns, dim3(hash_blocks), dim3(256 * kHashRowLanes), 0, stream,
-                          dfa_trans, Q, dead_state, ws.partial, tune.weak_hash, ws.meta, ws.gcount,
+                          dfa_trans, Q, dead_state, ws.partial, tune.weak_hash, ws.meta,
                           ws.count2, ws.cursor2, ws.row_ctr, status_word) != cudaSuccess)
         return FSM_ERR_CUDA;
     // prepare_all: blocks share the table rows and the tokens
@@ -100,7 +100,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
         if (launch_overlapped(k, dim3(prep_blocks), dim3(kPrepThreads), key_smem, stream, dfa_trans,
                               vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
                               ws.partial, hash_blocks, ws.meta, ws.cls, static_cast<int32_t*>(ws.table),
-                              tok_cls, ws.tok_len, live, ws.gcount, count2, planes,
+                              tok_cls, ws.tok_len, live, count2, planes,
                               bucket ? ws.tok_head : nullptr, status_word) != cudaSuccess)
             return FSM_ERR_CUDA;
     } else {
@@ -111,7 +111,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
         if (launch_overlapped(k, dim3(prep_blocks), dim3(kPrepThreads), key_smem, stream, dfa_trans,
                               vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
                               ws.partial, hash_blocks, ws.meta, ws.cls, static_cast<uint16_t*>(ws.table),
-                              tok_cls, ws.tok_len, live, ws.gcount, count2, planes,
+                              tok_cls, ws.tok_len, live, count2, planes,
                               bucket ? ws.tok_head : nullptr, status_word) != cudaSuccess)
             return FSM_ERR_CUDA;
     }

@@ -60,14 +60,13 @@ __device__ __forceinline__ bool stage_table(const WalkParams& p, TabT* stab, uin
 // ---------------------------------------------------------------------------------------
 // Bitmask words of the one-byte tokens (and zeros elsewhere).  Block (x, y): the 128
 // bitmask words 128x .. 128x+127 of the rows 8y + warp, 8y + warp + 8 gridDim.y, ...; those
-// words of the first 64 planes sit in shared memory; lane l handles words l, l+32, l+64,
-// l+96.
+// words of the first 64 planes sit in shared memory; lane l handles words 4l .. 4l+3.
 constexpr int kObThreads = 256;
 constexpr int kObWords = 128;
 constexpr int kObSmemClasses = 64;  // planes of further classes are read through the cache
 
 __global__ void __launch_bounds__(kObThreads) mask_onebyte(const WalkParams p) {
-    __shared__ uint32_t s_pl[kObSmemClasses * kObWords];  // planes of the first classes
+    __shared__ __align__(16) uint32_t s_pl[kObSmemClasses * kObWords];  // planes of the first classes
     __shared__ uint8_t s_live[kObThreads / 32][256];      // classes read by the warp's row
     if (p.meta->any_bad != 0) {
         // exact fallback: every token walked through the uncompressed table
@@ -96,29 +95,43 @@ __global__ void __launch_bounds__(kObThreads) mask_onebyte(const WalkParams p) {
             nlive += __popc(m);
         }
         __syncwarp();
-        uint32_t acc[kObWords / 32] = {0, 0, 0, 0};
+        // lane l holds words 4l .. 4l+3 of the block's 128
+        uint4 acc = make_uint4(0, 0, 0, 0);
+        const int wl = w0 + 4 * lane;
         for (int j = 0; j < nlive; ++j) {
             const int c = mine[j];
+            uint4 v;
             if (c < kObSmemClasses) {
-                const uint32_t* pl = s_pl + c * kObWords + lane;
-#pragma unroll
-                for (int i = 0; i < kObWords / 32; ++i) acc[i] |= pl[32 * i];
+                v = *reinterpret_cast<const uint4*>(s_pl + c * kObWords + 4 * lane);
             } else {
-                const uint32_t* pl = p.planes + static_cast<size_t>(c) * p.G + w0 + lane;
-#pragma unroll
-                for (int i = 0; i < kObWords / 32; ++i)
-                    if (w0 + lane + 32 * i < p.G) acc[i] |= __ldg(pl + 32 * i);
+                const uint32_t* pl = p.planes + static_cast<size_t>(c) * p.G + wl;
+                v.x = wl < p.G ? __ldg(pl) : 0u;
+                v.y = wl + 1 < p.G ? __ldg(pl + 1) : 0u;
+                v.z = wl + 2 < p.G ? __ldg(pl + 2) : 0u;
+                v.w = wl + 3 < p.G ? __ldg(pl + 3) : 0u;
             }
+            acc.x |= v.x;
+            acc.y |= v.y;
+            acc.z |= v.z;
+            acc.w |= v.w;
         }
-        if (eos_word >= 0 && eos_word < kObWords && (eos_word & 31) == lane && q != p.dead && p.accept[q]) {
-#pragma unroll
-            for (int i = 0; i < kObWords / 32; ++i)
-                if ((eos_word >> 5) == i) acc[i] |= 1u << (p.eos_id & 31);
+        if (eos_word >= 0 && eos_word < kObWords && (eos_word >> 2) == lane && q != p.dead && p.accept[q]) {
+            const uint32_t bit = 1u << (p.eos_id & 31);
+            const int k = eos_word & 3;
+            acc.x |= k == 0 ? bit : 0u;
+            acc.y |= k == 1 ? bit : 0u;
+            acc.z |= k == 2 ? bit : 0u;
+            acc.w |= k == 3 ? bit : 0u;
         }
-        uint32_t* mrow = p.mask + static_cast<size_t>(r) * p.G + w0 + lane;
-#pragma unroll
-        for (int i = 0; i < kObWords / 32; ++i)
-            if (w0 + lane + 32 * i < p.G) mrow[32 * i] = acc[i];
+        uint32_t* mrow = p.mask + static_cast<size_t>(r) * p.G + wl;
+        if (wl + 3 < p.G && (reinterpret_cast<uintptr_t>(mrow) & 15) == 0) {
+            *reinterpret_cast<uint4*>(mrow) = acc;
+        } else {
+            if (wl < p.G) mrow[0] = acc.x;
+            if (wl + 1 < p.G) mrow[1] = acc.y;
+            if (wl + 2 < p.G) mrow[2] = acc.z;
+            if (wl + 3 < p.G) mrow[3] = acc.w;
+        }
         __syncwarp();  // the list is rewritten for the next row
     }
 }

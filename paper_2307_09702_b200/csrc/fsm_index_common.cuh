@@ -36,7 +36,6 @@ struct Workspace {
     // sparse walk: tokens sorted by bucket key
     uint4* srec;         // [N] {min(len,17), class of byte 1..15}
     int32_t* sid;        // [N] token id, same order as srec
-    int32_t* gcount;     // [256] tokens per first-byte class
     int32_t* gstart;     // [257] first sorted position of each first-byte class
     int32_t* row_ctr;    // [1] rows handed out by the sparse walk beyond the first one per CTA
     int32_t* count2;     // [kKeys] tokens per (first class, second key)
@@ -85,7 +84,6 @@ inline Workspace carve(void* base, int32_t Q, int32_t N) {
     w.tok_len = tokens ? tokens + G32 * sizeof(uint4) : nullptr;
     w.srec = reinterpret_cast<uint4*>(tokens);
     w.sid = reinterpret_cast<int32_t*>(tokens ? tokens + srec_bytes : nullptr);
-    w.gcount = reinterpret_cast<int32_t*>(take(256 * sizeof(int32_t)));
     w.gstart = reinterpret_cast<int32_t*>(take(257 * sizeof(int32_t)));
     w.row_ctr = reinterpret_cast<int32_t*>(take(sizeof(int32_t)));
     w.count2 = reinterpret_cast<int32_t*>(take(kKeys * sizeof(int32_t)));

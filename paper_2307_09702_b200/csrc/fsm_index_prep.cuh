@@ -22,7 +22,7 @@ constexpr int kHashRowLanes = 4;
 __global__ void __launch_bounds__(256 * kHashRowLanes)
 hash_columns(const int32_t* __restrict__ trans, int32_t Q, int32_t dead,
              uint64_t* __restrict__ partial, int weak, IndexMeta* meta,
-             int32_t* __restrict__ gcount, int32_t* __restrict__ count2,
+             int32_t* __restrict__ count2,
              int32_t* __restrict__ cursor2, int32_t* __restrict__ row_ctr, int32_t* status) {
     __shared__ uint64_t part[kHashRowLanes][256];
     const int b = threadIdx.x & 255, rl = threadIdx.x >> 8;
@@ -45,7 +45,6 @@ hash_columns(const int32_t* __restrict__ trans, int32_t Q, int32_t dead,
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < kKeys; i += gridDim.x * blockDim.x) {
         count2[i] = 0;
         cursor2[i] = 0;
-        if (i < 256) gcount[i] = 0;
     }
     part[rl][b] = h;
     const int any_bad = __syncthreads_or(bad);
@@ -141,14 +140,12 @@ prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab
             int32_t dead, int32_t eos_id, const uint64_t* partial, int nparts,
             IndexMeta* meta, uint8_t* __restrict__ cls_out, TabT* __restrict__ table,
             uint4* __restrict__ tok_cls, uint8_t* __restrict__ tok_len,
-            uint32_t* __restrict__ live, int32_t* __restrict__ gcount,
-            int32_t* __restrict__ count2, uint32_t* __restrict__ planes,
+            uint32_t* __restrict__ live, int32_t* __restrict__ count2, uint32_t* __restrict__ planes,
             uint16_t* __restrict__ tok_head, int32_t* status) {
     extern __shared__ int s_cnt[];  // [kKeys] when keys are counted
     __shared__ ClassScratch cs;
     __shared__ uint8_t s_cls[256], s_rep[256];
     __shared__ int32_t rows[kPrepRows][256];
-    __shared__ int hist[256];
     const int tid = threadIdx.x;
     // What does not depend on the classes is fetched first: the block's first pass of table
     // rows and of tokens.
@@ -242,7 +239,6 @@ prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab
         const int nkeys = two ? kKeys : 256;
         const int W = (N + 31) / 32;
         for (int i = tid; i < nkeys; i += kPrepThreads) s_cnt[i] = 0;
-        if (tid < 256) hist[tid] = 0;
         bool bad = bad_tok;
         for (int chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
             // bucket walk: plane c holds the bits of the one-byte tokens of class c; the
@@ -260,10 +256,7 @@ prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab
             const TokenInfo t = token_classify(raw, s_cls);
             if (tok_head != nullptr && v < N)  // first byte and length, for the compressed rows
                 tok_head[v] = static_cast<uint16_t>(raw.b0 | (static_cast<uint32_t>(raw.len) << 8));
-            if (t.len > 0) {
-                atomicAdd(&hist[t.first], 1);
-                atomicAdd(&s_cnt[bucket_key(two, t.first, t.second_key)], 1);
-            }
+            if (t.len > 0) atomicAdd(&s_cnt[bucket_key(two, t.first, t.second_key)], 1);
             if (planes != nullptr) {
                 const bool one = t.len == 1;
                 const uint32_t peers = __match_any_sync(kFullWarp, one ? t.first : 0xFFFF);
@@ -274,7 +267,6 @@ prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab
         if (__syncthreads_or(bad) && tid == 0) raise_flag(status, FSM_FLAG_OFFSETS);
         for (int i = tid; i < nkeys; i += kPrepThreads)
             if (s_cnt[i] > 0) atomicAdd(&count2[i], s_cnt[i]);
-        if (tid < 256 && hist[tid] > 0) atomicAdd(&gcount[tid], hist[tid]);
     }
 }
 
