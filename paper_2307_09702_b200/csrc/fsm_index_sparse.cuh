@@ -95,12 +95,14 @@ struct SurvivorSink {
 // One chunk: up to 32 tokens of a bucket (lane = token).  chunk_load fetches the lane's
 // record and token id; chunk_finish walks the rest of the token from state `s` (after
 // the DEPTH bytes the bucket key covers) and appends a survivor to its slice's list.
+// `with_rec` is false for a bucket of one-byte tokens: nothing of such a token is left to
+// walk, so its record is not fetched.
 __device__ __forceinline__ void chunk_load(const WalkParams& p, int pos, int count, int lane,
-                                           uint4& rec, int32_t& id) {
-    rec = make_uint4(0, 0, 0, 0);
+                                           bool with_rec, uint4& rec, int32_t& id) {
+    rec = make_uint4(1, 0, 0, 0);  // length 1
     id = -1;
     if (lane < count) {
-        rec = __ldg(p.srec + pos + lane);
+        if (with_rec) rec = __ldg(p.srec + pos + lane);
         id = __ldg(p.sid + pos + lane);
     }
 }
@@ -231,7 +233,7 @@ __device__ __forceinline__ void walk_row(const WalkParams& p, const TabT* __rest
                 for (int i0 = 0; i0 < bn; i0 += 32) {
                     uint4 rec;
                     int32_t id;
-                    chunk_load(p, bstart + i0, bn - i0, lane, rec, id);
+                    chunk_load(p, bstart + i0, bn - i0, lane, true, rec, id);
                     chunk_finish_depth<TabT, FULL>(p, tab, Cs, sink, rec, id, bs, depth);
                 }
             }
@@ -245,7 +247,8 @@ constexpr int kPull = 2;
 
 template <typename TabT, bool FULL>
 __device__ __forceinline__ void walk_chunks(const WalkParams& p, const TabT* __restrict__ tab,
-                                            uint32_t Cs, const SurvivorSink<TabT>& sink) {
+                                            uint32_t Cs, bool two_level,
+                                            const SurvivorSink<TabT>& sink) {
     using D = Desc<TabT>;
     const int lane = threadIdx.x & 31;
     const int total = sink.ctrs[1];
@@ -261,7 +264,9 @@ __device__ __forceinline__ void walk_chunks(const WalkParams& p, const TabT* __r
         for (int k = 0; k < kPull; ++k) {
             const bool have = i + k < total;
             d[k] = sink.descs[have ? i + k : i];
-            chunk_load(p, D::start(d[k]), have ? D::count(d[k]) : 0, lane, rec[k], id[k]);
+            // with two-level keys a bucket of depth 1 holds the one-byte tokens
+            chunk_load(p, D::start(d[k]), have ? D::count(d[k]) : 0, lane,
+                       !(two_level && D::depth(d[k]) == 1), rec[k], id[k]);
         }
 #pragma unroll
         for (int k = 0; k < kPull; ++k)
@@ -495,9 +500,9 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
         }
         if (sink.ctrs[3] == 0) {
             if (full)
-                walk_chunks<TabT, true>(p, stab, Cs, sink);
+                walk_chunks<TabT, true>(p, stab, Cs, two_level, sink);
             else
-                walk_chunks<TabT, false>(p, gtab, Cs, sink);
+                walk_chunks<TabT, false>(p, gtab, Cs, two_level, sink);
         } else {
             // more chunks than the list holds (a state that reads almost everything):
             // walk the buckets unit by unit instead
