@@ -209,14 +209,24 @@ __device__ __forceinline__ void mask_vector(uint32_t (&w)[NW], uint32_t bits) {
 
 // Pool of allowed entries of one warp.  Few entries of a vector are allowed (one in
 // eighteen in the benchmark's index), so scoring them lane by lane would run the draw with
-// most lanes idle; instead every lane appends its (logit, id) pairs to the warp's queue and
-// the warp scores 32 queued entries at a time.  kQueue holds the leftovers of one round
+// most lanes idle; instead every lane appends the ids of its allowed entries to the warp's
+// queue and the warp scores 32 queued entries at a time, each lane fetching its entry's
+// logit again by id (the row was read a moment ago: an L2 hit, and one instruction instead
+// of picking the value out of the vector's registers).  kQueue holds the leftovers of one round
 // (< 32) plus every entry of one 32-byte vector per lane (at most 16 bf16 values).
 constexpr int kQueue = 32 + 16 * 32;
 struct WarpQueue {
-    float x[kQueue];
     int id[kQueue];
 };
+
+// The logit of token `id` as fp32 (allowed entries are the same in the input and in the
+// masked output, so reading the input is right even while the row is being rewritten).
+template <typename T>
+__device__ __forceinline__ float logit_of(const T* in, int id) {
+    const T raw = in[id];
+    return sizeof(T) == 4 ? __uint_as_float(static_cast<uint32_t>(raw))
+                          : __uint_as_float(static_cast<uint32_t>(raw) << 16);
+}
 
 // The queues of a CTA; the greedy variant has none.
 template <bool SAMPLE> struct QueueStore {
@@ -229,12 +239,10 @@ template <> struct QueueStore<false> {
     __device__ static WarpQueue* get() { return nullptr; }
 };
 
-// All 32 lanes call this with their vector (bits == 0: nothing to add).
-template <typename T, int NW>
-__device__ __forceinline__ void pool_vector(const uint32_t (&w)[NW], uint32_t bits, int first_id,
-                                            uint32_t row, const StepParams& p, WarpQueue& q, int& qn,
-                                            Best& best) {
-    constexpr int PW = Elem<T>::kPerWord;
+// All 32 lanes call this with the allowed bits of their vector (0: nothing to add).
+template <typename T>
+__device__ __forceinline__ void pool_vector(uint32_t bits, int first_id, const T* in, uint32_t row,
+                                            const StepParams& p, WarpQueue& q, int& qn, Best& best) {
     const int lane = threadIdx.x & 31;
     const int mine = __popc(bits);
     int incl = mine;
@@ -246,35 +254,20 @@ __device__ __forceinline__ void pool_vector(const uint32_t (&w)[NW], uint32_t bi
     const int total = __shfl_sync(kFullWarp, incl, 31);
     if (total == 0) return;
     int at = qn + incl - mine;
-    uint32_t todo = bits;
-    while (todo) {
-        const int j = __ffs(todo) - 1;
-        todo &= todo - 1;
-        uint32_t word = w[0];
-#pragma unroll
-        for (int i = 1; i < NW; ++i) word = (j / PW == i) ? w[i] : word;
-        q.x[at] = Elem<T>::get(word, j % PW);
-        q.id[at] = first_id + j;
-        ++at;
-    }
+    for (uint32_t todo = bits; todo != 0; todo &= todo - 1) q.id[at++] = first_id + __ffs(todo) - 1;
     qn += total;
     __syncwarp();
     int head = 0;
-    for (; qn - head >= 32; head += 32)
-        take_better(best, gumbel_score(q.x[head + lane], q.id[head + lane], row, p), q.id[head + lane]);
+    for (; qn - head >= 32; head += 32) {
+        const int id = q.id[head + lane];
+        take_better(best, gumbel_score(logit_of(in, id), id, row, p), id);
+    }
     if (head > 0) {  // leftovers to the front
         const int rem = qn - head;
-        float x = 0.0f;
         int id = 0;
-        if (lane < rem) {
-            x = q.x[head + lane];
-            id = q.id[head + lane];
-        }
+        if (lane < rem) id = q.id[head + lane];
         __syncwarp();
-        if (lane < rem) {
-            q.x[lane] = x;
-            q.id[lane] = id;
-        }
+        if (lane < rem) q.id[lane] = id;
         qn = rem;
     }
     __syncwarp();
@@ -341,7 +334,7 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
                     const int vi = g0 + (h + u) * nthreads;
-                    if (SAMPLE) pool_vector<T, 8>(v[u].w, bits[h + u], vi * EPV, row, p, queue, qn, best);
+                    if (SAMPLE) pool_vector<T>(bits[h + u], vi * EPV, in, row, p, queue, qn, best);
                     if (vi < nvec) {
                         if (bits[h + u] != 0) {
                             if (SAMPLE)
@@ -357,9 +350,10 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
                 }
             }
         }
-        if (SAMPLE && static_cast<int>(threadIdx.x & 31) < qn)  // what is left in the pool
-            take_better(best, gumbel_score(queue.x[threadIdx.x & 31], queue.id[threadIdx.x & 31], row, p),
-                        queue.id[threadIdx.x & 31]);
+        if (SAMPLE && static_cast<int>(threadIdx.x & 31) < qn) {  // what is left in the pool
+            const int id = queue.id[threadIdx.x & 31];
+            take_better(best, gumbel_score(logit_of(in, id), id, row, p), id);
+        }
         done = nvec * EPV;
     } else {
         const int nvec = p.N / EPH;
