@@ -307,9 +307,10 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
     if (wide) {
         // Per thread and pass: the bitmask bits of kGroup vectors are fetched first (one
         // round trip to L2), then the vectors are streamed kUnroll at a time - every needed
-        // logits load of a batch is issued before any arithmetic, so that several 32-byte
-        // loads are in flight per thread.
-        constexpr int kUnroll = 4, kGroup = 8;
+        // logits load of a batch is issued before any arithmetic.  Two loads in flight per
+        // thread keep the kernel at 64 registers (four CTAs per SM), which measured faster
+        // than four or eight loads at 80 to 160 registers.
+        constexpr int kUnroll = 2, kGroup = 4;
         const int nvec = p.N / EPV;
         constexpr uint32_t kBitsMask = (EPV == 32) ? 0xFFFFFFFFu : ((1u << EPV) - 1u);
         WarpQueue& queue = QueueStore<SAMPLE>::get()[SAMPLE ? (threadIdx.x >> 5) : 0];
@@ -519,13 +520,14 @@ int step_impl(const void* logits_in, void* logits_out, int32_t logits_dtype, int
     if (!dev.ok) return FSM_ERR_CUDA;
     if (dev.cc_major != 10) return FSM_ERR_DEVICE;
 
-    // CTAs per row: enough CTAs to fill the device several times over, but at least
-    // a few vectors per thread.
+    // CTAs per row: the smallest cluster that gives at least three CTAs per SM (four fit, by
+    // registers, so the whole grid is resident at once), but at least a few vectors per
+    // thread.  Measured at B = 256, N = 128,256, bf16: 32.9 / 26.9 / 29.3 us with 1 / 2 / 4.
     int k = tunables().mask_cluster;
     if (k != 1 && k != 2 && k != 4 && k != 8) {
         k = 1;
         const int64_t vectors = static_cast<int64_t>(N) * esize / 32;
-        while (k < 8 && static_cast<int64_t>(B) * k < 6LL * dev.sm_count &&
+        while (k < 8 && static_cast<int64_t>(B) * k < 3LL * dev.sm_count &&
                vectors / (2 * k * kStepThreads) >= 2)
             k *= 2;
     }
