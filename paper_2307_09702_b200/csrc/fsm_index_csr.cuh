@@ -72,14 +72,14 @@ csr_scan(const int32_t* __restrict__ row_count, int32_t nrows, int64_t* __restri
 
 constexpr int kFillThreads = 128;
 constexpr int kFillWarps = kFillThreads / 32;
-constexpr int kLongCap = 512;  // tokens set aside for a walk before the warp walks them
+constexpr int kLongCap = 256;  // tokens set aside for a walk before the warp walks them
 
 __global__ void __launch_bounds__(kFillThreads)
 csr_fill(const WalkParams p, const uint16_t* __restrict__ tok_head,
          const int64_t* __restrict__ row_offsets, int32_t* __restrict__ csr_tokens,
          int32_t* __restrict__ csr_next, int64_t capacity) {
     __shared__ int wsum[kFillWarps], wfront[kFillWarps];
-    __shared__ int s_ids[kFillWarps][1024];        // token ids of 32 bitmask words, in order
+    __shared__ uint16_t s_ids[kFillWarps][1024];   // tokens of 32 bitmask words, in order (id - 32 * first word)
     __shared__ int2 s_long[kFillWarps][kLongCap];  // (entry position - row start, token) to walk
     const int nrows = p.q_end - p.q_begin;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -89,7 +89,7 @@ csr_fill(const WalkParams p, const uint16_t* __restrict__ tok_head,
     const int b0 = min(p.G, static_cast<int>(blockIdx.y) * bper), b1 = min(p.G, b0 + bper);
     const int wper = ((b1 - b0 + kFillWarps - 1) / kFillWarps + 31) / 32 * 32;
     const int w0 = min(b1, b0 + warp * wper), w1 = min(b1, w0 + wper);
-    int* ids = s_ids[warp];
+    uint16_t* ids = s_ids[warp];
     int2* longs = s_long[warp];
     for (int r = blockIdx.x; r < nrows; r += gridDim.x) {
         const int q = p.q_begin + r;
@@ -137,7 +137,7 @@ csr_fill(const WalkParams p, const uint16_t* __restrict__ tok_head,
             const int total = __shfl_sync(kFullWarp, incl, 31);
             int k = incl - cnt;
             while (bits) {
-                ids[k++] = wi * 32 + __ffs(bits) - 1;
+                ids[k++] = static_cast<uint16_t>(lane * 32 + __ffs(bits) - 1);
                 bits &= bits - 1;
             }
             __syncwarp();
@@ -148,7 +148,7 @@ csr_fill(const WalkParams p, const uint16_t* __restrict__ tok_head,
                 bool walk = false;
                 int v = 0;
                 if (j < total) {
-                    v = ids[j];
+                    v = base * 32 + ids[j];
                     const uint32_t head = __ldg(tok_head + v);
                     uint32_t s = q;  // EOS keeps the state
                     walk = v != p.eos_id && (head >> 8) != 1;
