@@ -523,11 +523,15 @@ int step_impl(const void* logits_in, void* logits_out, int32_t logits_dtype, int
     // CTAs per row: the smallest cluster that gives at least three CTAs per SM (four fit, by
     // registers, so the whole grid is resident at once), but at least a few vectors per
     // thread.  Measured at B = 256, N = 128,256, bf16: 32.9 / 26.9 / 29.3 us with 1 / 2 / 4.
+    // The categorical draw is bound by instruction issue and its CTAs differ in length (the
+    // work follows the allowed tokens), so it takes CTAs half as long, which fill the SMs
+    // more evenly as they come and go: 72.1 / 52.0 / 46.7 / 47.0 us with 1 / 2 / 4 / 8.
     int k = tunables().mask_cluster;
     if (k != 1 && k != 2 && k != 4 && k != 8) {
         k = 1;
         const int64_t vectors = static_cast<int64_t>(N) * esize / 32;
-        while (k < 8 && static_cast<int64_t>(B) * k < 3LL * dev.sm_count &&
+        const int64_t ctas_wanted = (sample ? 6LL : 3LL) * dev.sm_count;
+        while (k < 8 && static_cast<int64_t>(B) * k < ctas_wanted &&
                vectors / (2 * k * kStepThreads) >= 2)
             k *= 2;
     }
