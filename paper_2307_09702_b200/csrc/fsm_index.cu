@@ -88,7 +88,8 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     if (prep_blocks > dev.sm_count) prep_blocks = dev.sm_count;
     uint4* tok_cls = sparse ? nullptr : ws.tok_cls;  // dense walk: token records
     int32_t* count2 = sparse ? ws.count2 : nullptr;  // work-avoiding walks: bucket keys
-    uint32_t* live = bucket ? ws.live : nullptr;
+    uint32_t* live = sparse ? ws.live : nullptr;  // bucket walk; row order of the row-wise walk
+    int32_t* row_order = sparse && !bucket ? ws.row_order : nullptr;
     uint32_t* planes = bucket ? ws.planes : nullptr;
     const size_t key_smem = sparse ? kKeys * sizeof(int) : 0;
     const size_t sort_smem = (kKeysPad + kKeys) * sizeof(int);
@@ -120,10 +121,10 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
                                  static_cast<int>(sort_smem)) != cudaSuccess)
             return FSM_ERR_CUDA;
         const int sort_blocks = nchunks < dev.sm_count ? nchunks : dev.sm_count;
-        if (launch_overlapped(sort_all, dim3(sort_blocks), dim3(kPrepThreads), sort_smem, stream,
-                              vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id, ws.meta, ws.cls,
-                              ws.count2, ws.cursor2, ws.start2, ws.gstart, ws.srec,
-                              ws.sid) != cudaSuccess)
+        if (launch_overlapped(sort_all, dim3(sort_blocks + (row_order ? 1 : 0)), dim3(kPrepThreads),
+                              sort_smem, stream, vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id,
+                              ws.meta, ws.cls, ws.count2, ws.cursor2, ws.start2, ws.gstart, ws.srec,
+                              ws.sid, live, q_begin, q_end, row_order) != cudaSuccess)
             return FSM_ERR_CUDA;
     }
     if (cudaGetLastError() != cudaSuccess) return FSM_ERR_CUDA;
@@ -149,6 +150,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     p.sid = ws.sid;
     p.planes = ws.planes;
     p.live = ws.live;
+    p.row_order = row_order;
     p.gstart = ws.gstart;
     p.count2 = ws.count2;
     p.start2 = ws.start2;

@@ -47,6 +47,7 @@ struct Workspace {
     uint32_t* live;      // [Q][8] bit c: state reads class c
     int32_t* row_count;  // [Q] allowed tokens per row (compressed-row build)
     uint16_t* tok_head;  // [N] first byte | min(length, 255) << 8 of every token
+    int32_t* row_order;  // [Q] rows of the row-wise walk, most candidate tokens first
     size_t bytes;        // everything above
     size_t dense_bytes;  // the part in front of `survivors`: enough for the dense walk
 };
@@ -97,6 +98,7 @@ inline Workspace carve(void* base, int32_t Q, int32_t N) {
     w.live = reinterpret_cast<uint32_t*>(take(static_cast<size_t>(Q) * 8 * sizeof(uint32_t)));
     w.row_count = reinterpret_cast<int32_t*>(take(static_cast<size_t>(Q) * sizeof(int32_t)));
     w.tok_head = reinterpret_cast<uint16_t*>(take(static_cast<size_t>(N) * sizeof(uint16_t)));
+    w.row_order = reinterpret_cast<int32_t*>(take(static_cast<size_t>(Q) * sizeof(int32_t)));
     w.bytes = off;
     return w;
 }
@@ -124,6 +126,7 @@ struct WalkParams {
     // bucket walk
     const uint32_t* planes;
     const uint32_t* live;
+    const int32_t* row_order;  // row-wise walk: rows in the order they are handed out, or null
     // outputs
     uint32_t* mask;
     void* next;

@@ -280,12 +280,14 @@ prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab
 // record keeps the length and the classes of bytes 1..15; `sid` holds the token id.
 constexpr int kScanPer = (kKeys + kPrepThreads - 1) / kPrepThreads;  // keys per thread
 constexpr int kKeysPad = kScanPer * kPrepThreads;
+constexpr int kOrderBuckets = 2048;  // candidate-count buckets of the row order
 
 __global__ void __launch_bounds__(kPrepThreads)
 sort_all(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vocab_offsets,
          int64_t vocab_nbytes, int32_t N, int32_t eos_id, const IndexMeta* meta,
          const uint8_t* cls, const int32_t* count2, int32_t* cursor2, int32_t* __restrict__ start2,
-         int32_t* __restrict__ gstart, uint4* __restrict__ srec, int32_t* __restrict__ sid) {
+         int32_t* __restrict__ gstart, uint4* __restrict__ srec, int32_t* __restrict__ sid,
+         const uint32_t* live, int32_t q_begin, int32_t q_end, int32_t* row_order) {
     extern __shared__ int s_sort[];  // s_start[kKeysPad], s_cnt[kKeys]
     int* s_start = s_sort;
     int* s_cnt = s_sort + kKeysPad;
@@ -336,6 +338,57 @@ sort_all(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vo
 #pragma unroll
     for (int j = 0; j < kScanPer; ++j) s_start[tid * kScanPer + j] = before + incl - sum + local[j];
     __syncthreads();
+    // With a row order asked for, the last block of the grid sorts no tokens: it ranks the
+    // states by the number of tokens that start with a byte they read (the candidates the
+    // row-wise walk has to look at, between none and most of the vocabulary), largest first.
+    // Rows handed out in that order leave the CTAs of the walk finishing together; in
+    // index order a CTA that draws a long row last keeps the kernel waiting.
+    const int sort_grid = static_cast<int>(gridDim.x) - (row_order != nullptr ? 1 : 0);
+    if (row_order != nullptr && static_cast<int>(blockIdx.x) == sort_grid) {
+        __shared__ int s_group[256];  // tokens per first-byte class
+        if (tid < 256) {
+            const int stride = two ? kKeyStride : 1, groups = two ? kKeyStride : 256;
+            const int g0 = tid < groups ? s_start[tid * stride] : total;
+            const int g1 = tid + 1 < groups ? s_start[(tid + 1) * stride] : total;
+            s_group[tid] = g1 - g0;
+        }
+        for (int i = tid; i < kOrderBuckets; i += kPrepThreads) s_cnt[i] = 0;
+        __syncthreads();
+        const int nrows = q_end - q_begin;
+        auto bucket_of = [&](int r) {  // bucket 0 holds the heaviest rows
+            const uint32_t* lv = live + static_cast<size_t>(q_begin + r) * 8;
+            int64_t candidates = 0;
+            for (int w = 0; w < 8; ++w) {
+                uint32_t m = lv[w];
+                while (m) {
+                    candidates += s_group[w * 32 + __ffs(m) - 1];
+                    m &= m - 1;
+                }
+            }
+            const int64_t b = candidates * kOrderBuckets / (static_cast<int64_t>(N) + 1);
+            return kOrderBuckets - 1 - static_cast<int>(b < kOrderBuckets - 1 ? b : kOrderBuckets - 1);
+        };
+        for (int r = tid; r < nrows; r += kPrepThreads) atomicAdd(&s_cnt[bucket_of(r)], 1);
+        __syncthreads();
+        static_assert(kOrderBuckets == 2 * kPrepThreads, "two buckets per thread");
+        const int a0 = s_cnt[2 * tid], a1 = s_cnt[2 * tid + 1];
+        int inc2 = a0 + a1;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int o = __shfl_up_sync(kFullWarp, inc2, off);
+            if (lane >= off) inc2 += o;
+        }
+        __syncthreads();  // wsum is read by every thread above
+        if (lane == 31) wsum[warp] = inc2;
+        __syncthreads();
+        int front = 0;
+        for (int w = 0; w < warp; ++w) front += wsum[w];
+        s_cnt[2 * tid] = front + inc2 - a0 - a1;
+        s_cnt[2 * tid + 1] = front + inc2 - a1;
+        __syncthreads();
+        for (int r = tid; r < nrows; r += kPrepThreads) row_order[atomicAdd(&s_cnt[bucket_of(r)], 1)] = r;
+        return;
+    }
     if (blockIdx.x == 0) {
         for (int i = tid; i < nkeys; i += kPrepThreads) start2[i] = s_start[i];
         if (tid <= 256) {
@@ -349,7 +402,7 @@ sort_all(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vo
         }
     }
     const int nchunks = (N + kPrepTokens - 1) / kPrepTokens;
-    for (int chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
+    for (int chunk = blockIdx.x; chunk < nchunks; chunk += sort_grid) {
         __syncthreads();  // the previous pass is done with s_cnt
         for (int i = tid; i < nkeys; i += kPrepThreads) s_cnt[i] = 0;
         __syncthreads();

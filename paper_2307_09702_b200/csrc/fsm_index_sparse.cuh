@@ -467,7 +467,8 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
     sink.ctrs = s_ctrs;
 
     // Rows differ in cost (a state that reads the class of the space byte has three times
-    // the survivors), so after its first row a CTA takes rows from a global counter.
+    // the survivors), so after its first row a CTA takes rows from a global counter, and the
+    // rows come in the order of p.row_order: most candidate tokens first.
     //
     // Per row: walk the chunk list | barrier | assemble the row, then enumerate the next
     // row's chunks (no barrier in between: enumeration touches only the descriptor list
@@ -486,10 +487,12 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
     for (int i = threadIdx.x; i < nslices; i += kWalkThreads) counts[i] = 0;
     if (threadIdx.x < 8) s_ctrs[threadIdx.x] = 0;
     __syncthreads();
-    int r = blockIdx.x, par = 0;
-    if (r < nrows) enumerate(r, par);
+    auto row_at = [&](int i) { return p.row_order != nullptr ? __ldg(p.row_order + i) : i; };
+    int at = blockIdx.x, par = 0;  // position in the order
+    int r = at < nrows ? row_at(at) : nrows;
+    if (at < nrows) enumerate(r, par);
     __syncthreads();  // the chunk list of the first row is complete
-    while (r < nrows) {
+    while (at < nrows) {
         const int q = p.q_begin + r;
         OutT* nrow = HAS_OUT ? static_cast<OutT*>(p.next) + static_cast<size_t>(r) * p.N : nullptr;
         uint32_t* mrow = p.mask + static_cast<size_t>(r) * p.G;
@@ -515,11 +518,11 @@ walk_sparse(const WalkParams p, typename Entry<TabT>::type* scratch, uint32_t ta
                 walk_row<TabT, false, false>(p, gtab, C, Cs, two_level, s_gstart, sink, q);
         }
         __syncthreads();  // every survivor of the row is in its list (stores visible CTA-wide)
-        const int next_row = s_next_row[par ^ 1];
+        at = s_next_row[par ^ 1];
         assemble_row<TabT, OutT, HAS_OUT>(p, sink, stage, mwords, nslices, q, nrow, mrow);
-        if (next_row < nrows) enumerate(next_row, par ^ 1);
+        r = at < nrows ? row_at(at) : nrows;
+        if (at < nrows) enumerate(r, par ^ 1);
         __syncthreads();  // slice counters cleared, next chunk list complete
-        r = next_row;
         par ^= 1;
     }
 }
