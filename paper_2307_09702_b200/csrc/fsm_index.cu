@@ -90,6 +90,8 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     int32_t* count2 = sparse ? ws.count2 : nullptr;  // work-avoiding walks: bucket keys
     uint32_t* live = sparse ? ws.live : nullptr;  // bucket walk; row order of the row-wise walk
     int32_t* row_order = sparse && !bucket ? ws.row_order : nullptr;
+    // (the ranking of the windows counts them in kKeys words of shared memory)
+    int32_t* win_order = bucket && sparse && (N + 31) / 32 <= kKeys ? ws.win_order : nullptr;
     uint32_t* planes = bucket ? ws.planes : nullptr;
     const size_t key_smem = sparse ? kKeys * sizeof(int) : 0;
     const size_t sort_smem = (kKeysPad + kKeys) * sizeof(int);
@@ -121,10 +123,10 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
                                  static_cast<int>(sort_smem)) != cudaSuccess)
             return FSM_ERR_CUDA;
         const int sort_blocks = nchunks < dev.sm_count ? nchunks : dev.sm_count;
-        if (launch_overlapped(sort_all, dim3(sort_blocks + (row_order ? 1 : 0)), dim3(kPrepThreads),
+        if (launch_overlapped(sort_all, dim3(sort_blocks + (row_order || win_order ? 1 : 0)), dim3(kPrepThreads),
                               sort_smem, stream, vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id,
                               ws.meta, ws.cls, ws.count2, ws.cursor2, ws.start2, ws.gstart, ws.srec,
-                              ws.sid, live, q_begin, q_end, row_order) != cudaSuccess)
+                              ws.sid, live, q_begin, q_end, row_order, win_order) != cudaSuccess)
             return FSM_ERR_CUDA;
     }
     if (cudaGetLastError() != cudaSuccess) return FSM_ERR_CUDA;
@@ -151,6 +153,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     p.planes = ws.planes;
     p.live = ws.live;
     p.row_order = row_order;
+    p.win_order = win_order;
     p.gstart = ws.gstart;
     p.count2 = ws.count2;
     p.start2 = ws.start2;

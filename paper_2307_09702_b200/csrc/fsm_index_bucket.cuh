@@ -153,16 +153,18 @@ __device__ __forceinline__ void bucket_tasks(const WalkParams& p, const TabT* __
     const int parts = (nrows + kStatesPerTask - 1) / kStatesPerTask;
     const int64_t ntasks = static_cast<int64_t>(nwin) * parts;
     // Tasks cost very differently (a window of rare keys holds many keys, each with its own
-    // scan of the states).  Task i of this CTA is task i * gridDim.x + blockIdx.x, so that
-    // neighbouring windows go to different SMs; inside the CTA warps draw from a counter.
+    // scan of the states).  The windows come in the order of p.win_order, most keys first;
+    // task i of this CTA is task i * gridDim.x + blockIdx.x of that order, so that every CTA
+    // gets the same mix, and inside the CTA warps draw from a counter, heaviest tasks first.
     while (true) {
         int i = 0;
         if (lane == 0) i = atomicAdd(s_next, 1);
         i = __shfl_sync(kFullWarp, i, 0);
         const int64_t t = static_cast<int64_t>(i) * gridDim.x + blockIdx.x;
         if (t >= ntasks) break;
-        const int win = static_cast<int>(t / parts);
-        const int part = static_cast<int>(t - static_cast<int64_t>(win) * parts);
+        const int wat = static_cast<int>(t / parts);
+        const int part = static_cast<int>(t - static_cast<int64_t>(wat) * parts);
+        const int win = p.win_order != nullptr ? __ldg(p.win_order + wat) : wat;
         const int pos = win * 32 + lane;
         uint4 rec = make_uint4(0, 0, 0, 0);
         int32_t id = -1;

@@ -48,6 +48,7 @@ struct Workspace {
     int32_t* row_count;  // [Q] allowed tokens per row (compressed-row build)
     uint16_t* tok_head;  // [N] first byte | min(length, 255) << 8 of every token
     int32_t* row_order;  // [Q] rows of the row-wise walk, most candidate tokens first
+    int32_t* win_order;  // [G] windows of 32 sorted tokens of the bucket walk, most keys first
     size_t bytes;        // everything above
     size_t dense_bytes;  // the part in front of `survivors`: enough for the dense walk
 };
@@ -99,6 +100,7 @@ inline Workspace carve(void* base, int32_t Q, int32_t N) {
     w.row_count = reinterpret_cast<int32_t*>(take(static_cast<size_t>(Q) * sizeof(int32_t)));
     w.tok_head = reinterpret_cast<uint16_t*>(take(static_cast<size_t>(N) * sizeof(uint16_t)));
     w.row_order = reinterpret_cast<int32_t*>(take(static_cast<size_t>(Q) * sizeof(int32_t)));
+    w.win_order = reinterpret_cast<int32_t*>(take(G32 / 32 * sizeof(int32_t)));
     w.bytes = off;
     return w;
 }
@@ -127,6 +129,7 @@ struct WalkParams {
     const uint32_t* planes;
     const uint32_t* live;
     const int32_t* row_order;  // row-wise walk: rows in the order they are handed out, or null
+    const int32_t* win_order;  // bucket walk: windows in the order they are handed out, or null
     // outputs
     uint32_t* mask;
     void* next;

@@ -287,7 +287,8 @@ sort_all(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vo
          int64_t vocab_nbytes, int32_t N, int32_t eos_id, const IndexMeta* meta,
          const uint8_t* cls, const int32_t* count2, int32_t* cursor2, int32_t* __restrict__ start2,
          int32_t* __restrict__ gstart, uint4* __restrict__ srec, int32_t* __restrict__ sid,
-         const uint32_t* live, int32_t q_begin, int32_t q_end, int32_t* row_order) {
+         const uint32_t* live, int32_t q_begin, int32_t q_end, int32_t* row_order,
+         int32_t* win_order) {
     extern __shared__ int s_sort[];  // s_start[kKeysPad], s_cnt[kKeys]
     int* s_start = s_sort;
     int* s_cnt = s_sort + kKeysPad;
@@ -343,7 +344,53 @@ sort_all(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vo
     // row-wise walk has to look at, between none and most of the vocabulary), largest first.
     // Rows handed out in that order leave the CTAs of the walk finishing together; in
     // index order a CTA that draws a long row last keeps the kernel waiting.
-    const int sort_grid = static_cast<int>(gridDim.x) - (row_order != nullptr ? 1 : 0);
+    const bool ordering = row_order != nullptr || win_order != nullptr;
+    const int sort_grid = static_cast<int>(gridDim.x) - (ordering ? 1 : 0);
+    if (win_order != nullptr && static_cast<int>(blockIdx.x) == sort_grid) {
+        // The same for the bucket walk: a window of 32 sorted tokens costs one scan of the
+        // states per (first class, second class) key in it, so the windows are ranked by the
+        // number of buckets of longer tokens that begin in them (0 to 32), most first; the
+        // bucket that reaches in from the window before is one more in nearly every window
+        // and is left out.  (Host: win_order only when the windows fit s_cnt.)
+        const int nwin = (total + 31) >> 5;
+        for (int i = tid; i < nwin; i += kPrepThreads) s_cnt[i] = 0;
+        __shared__ int s_hist[40];
+        if (tid < 40) s_hist[tid] = 0;
+        __syncthreads();
+        if (two) {
+            for (int key = tid; key < kKeys; key += kPrepThreads) {
+                const int st = s_start[key], en = s_start[key + 1];
+                if (en > st && key % kKeyStride != 0) atomicAdd(&s_cnt[st >> 5], 1);
+            }
+        }
+        __syncthreads();
+        // counting sort by that number, descending: the lanes of a warp that hold the same
+        // number find each other and reserve their places with one atomic
+        const int rounds = (nwin + kPrepThreads - 1) / kPrepThreads;
+        for (int pass = 0; pass < 2; ++pass) {
+            for (int it = 0; it < rounds; ++it) {
+                const int w = it * kPrepThreads + tid;
+                const int b = w < nwin ? 32 - min(s_cnt[w], 32) : 33;
+                const uint32_t m = __match_any_sync(kFullWarp, b);
+                const int leader = __ffs(m) - 1;
+                int base = 0;
+                if (lane == leader) base = atomicAdd(&s_hist[b], __popc(m));
+                base = __shfl_sync(kFullWarp, base, leader);
+                if (pass == 1 && w < nwin) win_order[base + __popc(m & ((1u << lane) - 1))] = w;
+            }
+            __syncthreads();
+            if (pass == 0 && tid == 0) {  // counts -> first positions
+                int run = 0;
+                for (int v = 0; v <= 33; ++v) {
+                    const int c = s_hist[v];
+                    s_hist[v] = run;
+                    run += c;
+                }
+            }
+            __syncthreads();
+        }
+        return;
+    }
     if (row_order != nullptr && static_cast<int>(blockIdx.x) == sort_grid) {
         __shared__ int s_group[256];  // tokens per first-byte class
         if (tid < 256) {
