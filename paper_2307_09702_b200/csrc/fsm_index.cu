@@ -70,8 +70,10 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     const bool want_sparse =
         tune.walk_algo == 2 || (tune.walk_algo == 0 && q_end - q_begin >= dev.sm_count);
     // Bitmask-only builds take the bucket walk (no dense rows to assemble).
+    // (like the row-wise walk it needs enough rows to fill the device)
     const bool bucket = next_state == nullptr && !dense_only &&
-                        (tune.walk_algo == 3 || tune.walk_algo == 0);
+                        (tune.walk_algo == 3 ||
+                         (tune.walk_algo == 0 && q_end - q_begin >= dev.sm_count));
     const bool sparse = (bucket || want_sparse) && !dense_only &&
                         (N + 255) / 256 <= kMaxSlices &&
                         sparse_table_offset<int32_t>(N) + 4096 <= static_cast<size_t>(dev.smem_optin - 2048);
@@ -285,13 +287,16 @@ extern "C" int fsm_index_build_csr(const int32_t* dfa_trans, const uint8_t* acce
     auto misaligned = [](const void* p, size_t a) { return reinterpret_cast<uintptr_t>(p) % a != 0; };
     if (misaligned(row_offsets, 8) || misaligned(csr_tokens, 4) || misaligned(csr_next, 4))
         return FSM_ERR_ALIGN;
+    if (Q <= 0 || N <= 0) return FSM_ERR_SHAPE;
+    Workspace ws = carve(workspace, Q, N);
+    uint16_t* dense_next = Q < kCsrDenseRows ? ws.csr_dense : nullptr;
     const int rc = build_rows_impl(dfa_trans, accept, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N,
-                                   dead_state, eos_id, 0, Q, allowed_mask, nullptr, FSM_STATE_I32,
-                                   workspace, workspace_bytes, status_word, cuda_stream, false);
+                                   dead_state, eos_id, 0, Q, allowed_mask, dense_next,
+                                   dense_next ? FSM_STATE_U16 : FSM_STATE_I32, workspace,
+                                   workspace_bytes, status_word, cuda_stream, false);
     if (rc != FSM_OK) return rc;
     const DeviceInfo& dev = device_info();
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    Workspace ws = carve(workspace, Q, N);
     WalkParams p = {};
     p.trans = dfa_trans;
     p.accept = accept;
@@ -312,7 +317,7 @@ extern "C" int fsm_index_build_csr(const int32_t* dfa_trans, const uint8_t* acce
     csr_scan<<<1, 1024, 0, stream>>>(ws.row_count, Q, row_offsets, capacity, status_word);
     const int fill_blocks = Q < 16 * dev.sm_count ? Q : 16 * dev.sm_count;
     const int fill_parts = p.G >= 8 * 32 * kFillWarps ? 8 : (p.G >= 4 * 32 * kFillWarps ? 4 : 1);
-    csr_fill<<<dim3(fill_blocks, fill_parts), kFillThreads, 0, stream>>>(p, ws.tok_head, row_offsets, csr_tokens, csr_next,
-                                                       capacity);
+    csr_fill<<<dim3(fill_blocks, fill_parts), kFillThreads, 0, stream>>>(
+        p, ws.tok_head, dense_next, row_offsets, csr_tokens, csr_next, capacity);
     return cudaGetLastError() == cudaSuccess ? FSM_OK : FSM_ERR_CUDA;
 }

@@ -235,9 +235,12 @@ __global__ void __launch_bounds__(kWalkThreads, 1) walk_buckets(const WalkParams
 template <typename TabT>
 cudaError_t launch_bucket(const WalkParams& p, int sms, cudaStream_t stream) {
     const int nrows = p.q_end - p.q_begin;
-    // mask_onebyte: 128 bitmask words per block column, rows spread over up to 16 block rows
+    // mask_onebyte: 128 bitmask words per block column, rows spread over the block rows
     const int ycap = (nrows + 7) / 8;
-    dim3 grid_a((p.G + kObWords - 1) / kObWords, ycap < 16 ? ycap : 16);
+    const int cols = (p.G + kObWords - 1) / kObWords;
+    int ymax = 5 * sms / cols;  // five blocks per SM (six fit): one even wave
+    if (ymax < 1) ymax = 1;
+    dim3 grid_a(cols, ycap < ymax ? ycap : ymax);
     cudaError_t e = launch_on(mask_onebyte, grid_a, dim3(kObThreads), 0, stream, p);
     if (e != cudaSuccess) return e;
     auto k1 = walk_buckets<TabT>;

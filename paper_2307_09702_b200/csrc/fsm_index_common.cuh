@@ -16,6 +16,7 @@ constexpr uint32_t kBulkChunk = 32768;  // bytes per bulk copy instruction (tabl
 constexpr int kKeyStride = 129;         // second-level keys per first-byte class (two-level sort)
 constexpr int kKeys = kKeyStride * kKeyStride;
 constexpr int kTwoLevelMaxC = 127;      // more classes than this: one-level buckets only
+constexpr int kCsrDenseRows = 256;      // smaller automata: compressed rows cut out of a dense table
 constexpr int kMaxSparseCtas = 160;     // CTAs of the sparse walk (one survivor scratch each)
 
 struct IndexMeta {
@@ -49,6 +50,8 @@ struct Workspace {
     uint16_t* tok_head;  // [N] first byte | min(length, 255) << 8 of every token
     int32_t* row_order;  // [Q] rows of the row-wise walk, most candidate tokens first
     int32_t* win_order;  // [G] windows of 32 sorted tokens of the bucket walk, most keys first
+    uint16_t* csr_dense; // [Q][N] end states of an automaton of fewer than kCsrDenseRows states
+                         // (compressed-row build: the rows are cut out of the dense table)
     size_t bytes;        // everything above
     size_t dense_bytes;  // the part in front of `survivors`: enough for the dense walk
 };
@@ -101,6 +104,8 @@ inline Workspace carve(void* base, int32_t Q, int32_t N) {
     w.tok_head = reinterpret_cast<uint16_t*>(take(static_cast<size_t>(N) * sizeof(uint16_t)));
     w.row_order = reinterpret_cast<int32_t*>(take(static_cast<size_t>(Q) * sizeof(int32_t)));
     w.win_order = reinterpret_cast<int32_t*>(take(G32 / 32 * sizeof(int32_t)));
+    w.csr_dense = reinterpret_cast<uint16_t*>(
+        take(Q < kCsrDenseRows ? static_cast<size_t>(Q) * N * sizeof(uint16_t) : 0));
     w.bytes = off;
     return w;
 }

@@ -9,6 +9,9 @@
 //              expanded into the list of their token ids (increasing), then lane = token:
 //              the end state of a one-byte token is delta(q, byte), the other tokens are
 //              collected and walked once more through the uncompressed table.
+// An automaton of fewer than kCsrDenseRows states (a typical regular expression) gives the
+// walks too few rows to spread over the SMs, and its rows are long: for it the dense table
+// is built into the workspace (16-bit states) and csr_fill copies the end states from it.
 #pragma once
 
 #include "fsm_index_common.cuh"
@@ -76,8 +79,8 @@ constexpr int kLongCap = 256;  // tokens set aside for a walk before the warp wa
 
 __global__ void __launch_bounds__(kFillThreads)
 csr_fill(const WalkParams p, const uint16_t* __restrict__ tok_head,
-         const int64_t* __restrict__ row_offsets, int32_t* __restrict__ csr_tokens,
-         int32_t* __restrict__ csr_next, int64_t capacity) {
+         const uint16_t* __restrict__ dense_next, const int64_t* __restrict__ row_offsets,
+         int32_t* __restrict__ csr_tokens, int32_t* __restrict__ csr_next, int64_t capacity) {
     __shared__ int wsum[kFillWarps], wfront[kFillWarps];
     __shared__ uint16_t s_ids[kFillWarps][1024];   // tokens of 32 bitmask words, in order (id - 32 * first word)
     __shared__ int2 s_long[kFillWarps][kLongCap];  // (entry position - row start, token) to walk
@@ -149,10 +152,15 @@ csr_fill(const WalkParams p, const uint16_t* __restrict__ tok_head,
                 int v = 0;
                 if (j < total) {
                     v = base * 32 + ids[j];
-                    const uint32_t head = __ldg(tok_head + v);
                     uint32_t s = q;  // EOS keeps the state
-                    walk = v != p.eos_id && (head >> 8) != 1;
-                    if (v != p.eos_id && !walk) s = clamp_state(__ldg(trow + (head & 0xFFu)), p.Q, p.dead);
+                    if (dense_next != nullptr) {  // small automaton: the dense table was built
+                        s = __ldg(dense_next + static_cast<size_t>(r) * p.N + v);
+                    } else {
+                        const uint32_t head = __ldg(tok_head + v);
+                        walk = v != p.eos_id && (head >> 8) != 1;
+                        if (v != p.eos_id && !walk)
+                            s = clamp_state(__ldg(trow + (head & 0xFFu)), p.Q, p.dead);
+                    }
                     if (row_at + at + j < capacity) {
                         csr_tokens[row_at + at + j] = v;
                         if (!walk) csr_next[row_at + at + j] = static_cast<int32_t>(s);
