@@ -40,7 +40,7 @@ SMEM_LOOKUP_BOUND = 148 * 32 * 1.965e9 / 1.157
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/
 # (walk_sparse_config3.md, mask_step_config5.md).  Set an entry to None when the kernel
 # changes and the capture has not been redone.
-NCU_TRAFFIC = {"walk_sparse": 508_000_000, "mask_step": 68_600_000}
+NCU_TRAFFIC = {"walk_sparse": 506_000_000, "mask_step": 68_600_000}
 # kernels of this library per timed step: hash_columns, prepare_all, sort_all, walk_sparse,
 # mask_step
 RING = 8
