@@ -4,7 +4,8 @@ import numpy as np
 import pytest
 import torch
 
-from fsm_inputs import f32_to_bf16_bits, make_config, random_class_dfa, start_states, vocab_from_strings
+from fsm_inputs import (bpe_like_vocab, f32_to_bf16_bits, make_config, random_class_dfa, start_states,
+                        vocab_from_strings)
 from oracle import fsm_oracle
 
 pytestmark = pytest.mark.gpu
@@ -62,6 +63,15 @@ def test_ragged_vocabularies_and_empty_rows(N):
     toks = [bytes(rng.integers(0, 256, size=rng.integers(0, 7)).tolist()) for _ in range(N)]
     vb, vo = vocab_from_strings(toks)
     check_csr(d.trans, d.accept, vb, vo, d.dead, N - 1)
+
+
+@pytest.mark.parametrize("n_live", [199, 255, 300])
+def test_automata_around_the_dense_table_threshold(n_live):
+    # under 256 states the rows are cut out of a dense table built into the workspace (by the
+    # row-wise walk once there is a row per SM), from 256 states on out of the bucket walk's bitmask
+    d, _ = random_class_dfa(n_live, n_live=n_live, n_classes=40, live_classes_per_state=9)
+    vb, vo = bpe_like_vocab(7, 5000, zero_length_ids=(4999,))
+    check_csr(d.trans, d.accept, vb, vo, d.dead, 4999)
 
 
 def test_capacity_too_small_is_flagged_and_offsets_stay_complete():
