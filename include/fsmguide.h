@@ -282,10 +282,12 @@ int guided_step_csr(const void* logits_in, void* logits_out, int32_t logits_dtyp
 #define FSM_TUNE_SMEM_TABLE_BYTES 4 /* cap on the shared-memory table tile; 0 = device maximum */
 #define FSM_PROFILE_WALK 5          /* non-zero: record a CUDA event pair around the walk
                                        kernel of every index build (see fsm_profile_read) */
-#define FSM_TUNE_WALK_ALGO 6        /* 0 = automatic, 1 = dense warp-tile walk, 2 = row-wise
-                                       work-avoiding walk, 3 = bucket walk (bitmask-only builds;
-                                       builds with a next-state table fall back to 1).  Same
-                                       results in every case */
+#define FSM_TUNE_WALK_ALGO 6        /* 0 = automatic (a build of at least one row per SM: 2
+                                       with a next-state table, 3 without; a smaller one: 1),
+                                       1 = dense warp-tile walk, 2 = row-wise work-avoiding
+                                       walk, 3 = bucket walk (bitmask-only builds; builds with
+                                       a next-state table fall back to 1).  Same results in
+                                       every case */
 int fsm_debug_set(int32_t key, int32_t value);
 
 /*
