@@ -314,10 +314,10 @@ extern "C" int fsm_index_build_csr(const int32_t* dfa_trans, const uint8_t* acce
     p.status = status_word;
     const int blocks = Q < 8 * dev.sm_count ? Q : 8 * dev.sm_count;
     csr_count<<<blocks, kCsrThreads, 0, stream>>>(allowed_mask, p.G, Q, ws.row_count);
-    csr_scan<<<1, 1024, 0, stream>>>(ws.row_count, Q, row_offsets, capacity, status_word);
+    csr_scan<<<1, 1024, 0, stream>>>(ws.row_count, Q, row_offsets, capacity, N, ws.row_order, status_word);
     const int fill_blocks = Q < 16 * dev.sm_count ? Q : 16 * dev.sm_count;
     const int fill_parts = p.G >= 8 * 32 * kFillWarps ? 8 : (p.G >= 4 * 32 * kFillWarps ? 4 : 1);
     csr_fill<<<dim3(fill_blocks, fill_parts), kFillThreads, 0, stream>>>(
-        p, ws.tok_head, dense_next, row_offsets, csr_tokens, csr_next, capacity);
+        p, ws.tok_head, dense_next, ws.row_order, row_offsets, csr_tokens, csr_next, capacity);
     return cudaGetLastError() == cudaSuccess ? FSM_OK : FSM_ERR_CUDA;
 }

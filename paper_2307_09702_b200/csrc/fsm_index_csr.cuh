@@ -20,6 +20,7 @@ namespace fsm {
 namespace {
 
 constexpr int kCsrThreads = 256;
+constexpr int kCsrRankBuckets = 1024;  // row-length buckets of csr_fill's row order
 
 __global__ void __launch_bounds__(kCsrThreads)
 csr_count(const uint32_t* __restrict__ mask, int32_t G, int32_t nrows, int32_t* __restrict__ row_count) {
@@ -43,9 +44,10 @@ csr_count(const uint32_t* __restrict__ mask, int32_t G, int32_t nrows, int32_t* 
 
 __global__ void __launch_bounds__(1024)
 csr_scan(const int32_t* __restrict__ row_count, int32_t nrows, int64_t* __restrict__ row_offsets,
-         int64_t capacity, int32_t* status) {
+         int64_t capacity, int32_t N, int32_t* __restrict__ row_order, int32_t* status) {
     __shared__ long long wsum[32];
     __shared__ long long carry;
+    __shared__ int s_rank[kCsrRankBuckets];
     if (threadIdx.x == 0) carry = 0;
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -71,6 +73,33 @@ csr_scan(const int32_t* __restrict__ row_count, int32_t nrows, int64_t* __restri
         row_offsets[nrows] = carry;
         if (carry > capacity) raise_flag(status, FSM_FLAG_CSR_OVERFLOW);
     }
+    // The rows in the order csr_fill takes them: longest first (counting sort by length), so
+    // that the blocks of the long rows do not start last.
+    auto bucket_of = [&](int r) {
+        const long long b = static_cast<long long>(row_count[r]) * kCsrRankBuckets / (static_cast<long long>(N) + 1);
+        return kCsrRankBuckets - 1 - static_cast<int>(b < kCsrRankBuckets - 1 ? b : kCsrRankBuckets - 1);
+    };
+    static_assert(kCsrRankBuckets == 1024, "one bucket per thread");
+    s_rank[threadIdx.x] = 0;
+    __syncthreads();
+    for (int r = threadIdx.x; r < nrows; r += 1024) atomicAdd(&s_rank[bucket_of(r)], 1);
+    __syncthreads();
+    {
+        const int mine = s_rank[threadIdx.x];
+        int incl = mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int o = __shfl_up_sync(kFullWarp, incl, off);
+            if (lane >= off) incl += o;
+        }
+        if (lane == 31) wsum[warp] = incl;
+        __syncthreads();
+        int before = 0;
+        for (int w = 0; w < warp; ++w) before += static_cast<int>(wsum[w]);
+        s_rank[threadIdx.x] = before + incl - mine;
+    }
+    __syncthreads();
+    for (int r = threadIdx.x; r < nrows; r += 1024) row_order[atomicAdd(&s_rank[bucket_of(r)], 1)] = r;
 }
 
 constexpr int kFillThreads = 128;
@@ -79,7 +108,8 @@ constexpr int kLongCap = 256;  // tokens set aside for a walk before the warp wa
 
 __global__ void __launch_bounds__(kFillThreads)
 csr_fill(const WalkParams p, const uint16_t* __restrict__ tok_head,
-         const uint16_t* __restrict__ dense_next, const int64_t* __restrict__ row_offsets,
+         const uint16_t* __restrict__ dense_next, const int32_t* __restrict__ row_order,
+         const int64_t* __restrict__ row_offsets,
          int32_t* __restrict__ csr_tokens, int32_t* __restrict__ csr_next, int64_t capacity) {
     __shared__ int wsum[kFillWarps], wfront[kFillWarps];
     __shared__ uint16_t s_ids[kFillWarps][1024];   // tokens of 32 bitmask words, in order (id - 32 * first word)
@@ -94,7 +124,8 @@ csr_fill(const WalkParams p, const uint16_t* __restrict__ tok_head,
     const int w0 = min(b1, b0 + warp * wper), w1 = min(b1, w0 + wper);
     uint16_t* ids = s_ids[warp];
     int2* longs = s_long[warp];
-    for (int r = blockIdx.x; r < nrows; r += gridDim.x) {
+    for (int ri = blockIdx.x; ri < nrows; ri += gridDim.x) {
+        const int r = row_order[ri];
         const int q = p.q_begin + r;
         const uint32_t* mrow = p.mask + static_cast<size_t>(r) * p.G;
         const int32_t* trow = p.trans + static_cast<size_t>(q) * 256;
