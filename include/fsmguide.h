@@ -98,8 +98,9 @@ size_t fsm_index_workspace_bytes(int32_t Q, int32_t N, int64_t vocab_nbytes);
  *                  fsm_index_workspace_bytes(Q, N, vocab_nbytes) bytes (the compressed
  *                  table, the token records and, for the work-avoiding walk, per-CTA
  *                  survivor lists of min(Q,160) * N entries: about 85 MB for 1,001
- *                  states and 128,256 tokens).  Contents on entry are irrelevant;
- *                  concurrent calls need separate workspaces.
+ *                  states and 128,256 tokens; for Q < 256 also Q * N 16-bit entries,
+ *                  from which fsm_index_build_csr cuts its rows).  Contents on entry
+ *                  are irrelevant; concurrent calls need separate workspaces.
  *   status_word    device int32 or NULL.
  *
  * fsm_index_build_rows builds only rows q_begin <= q < q_end, written to
