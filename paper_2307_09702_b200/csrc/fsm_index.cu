@@ -173,7 +173,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
         grid = q_end - q_begin;
     } else {
         const int64_t tasks = static_cast<int64_t>((q_end - q_begin + kChunk - 1) / kChunk) * G;
-        grid = (tasks + kWalkWarps - 1) / kWalkWarps;
+        grid = tasks;  // capped at one CTA per SM below; its warps take the tasks round-robin
     }
     if (grid > dev.sm_count) grid = dev.sm_count;
     if (sparse && grid > kMaxSparseCtas) grid = kMaxSparseCtas;

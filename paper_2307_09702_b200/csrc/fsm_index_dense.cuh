@@ -91,7 +91,9 @@ __global__ void __launch_bounds__(kWalkThreads, 1) walk(const WalkParams p) {
     const int cap_rows = max(kChunk, (static_cast<int>(tile_cap / row_bytes) - 3) / kChunk * kChunk);
     const int ntiles = full ? 1 : (nrows + cap_rows - 1) / cap_rows;
     const int lane = threadIdx.x & 31;
-    const int64_t wg = static_cast<int64_t>(blockIdx.x) * kWalkWarps + (threadIdx.x >> 5);
+    // warp w of CTA b starts at task w * gridDim.x + b: a build with fewer tasks than warps
+    // on the device still spreads over all the SMs
+    const int64_t wg = static_cast<int64_t>(threadIdx.x >> 5) * gridDim.x + blockIdx.x;
     const int64_t TW = static_cast<int64_t>(gridDim.x) * kWalkWarps;
 
     if (threadIdx.x == 0) {
