@@ -155,6 +155,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     p.planes = ws.planes;
     p.live = ws.live;
     p.row_order = row_order;
+    p.chunk = kChunk;
     p.win_order = win_order;
     p.gstart = ws.gstart;
     p.count2 = ws.count2;
@@ -172,7 +173,11 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     if (sparse) {
         grid = q_end - q_begin;
     } else {
-        const int64_t tasks = static_cast<int64_t>((q_end - q_begin + kChunk - 1) / kChunk) * G;
+        // States per warp task: fewer for a small build, until every warp of the device has
+        // two tasks (a task walks its states one after the other, so its length is latency).
+        auto tasks_with = [&](int c) { return static_cast<int64_t>((q_end - q_begin + c - 1) / c) * G; };
+        p.chunk = tasks_with(kChunk) < 2LL * dev.sm_count * kWalkWarps ? kSmallChunk : kChunk;
+        const int64_t tasks = tasks_with(p.chunk);
         grid = tasks;  // capped at one CTA per SM below; its warps take the tasks round-robin
     }
     if (grid > dev.sm_count) grid = dev.sm_count;

@@ -11,6 +11,7 @@ constexpr int kMaxCs = 264;             // bound on the row stride (256 classes 
 constexpr int kWalkThreads = 1024;
 constexpr int kWalkWarps = kWalkThreads / 32;
 constexpr int kChunk = 32;              // states per warp task (dense walk)
+constexpr int kSmallChunk = 8;          // the same for builds of few tasks
 constexpr int kInlineBytes = 16;        // token bytes kept in a 16-byte record
 constexpr uint32_t kBulkChunk = 32768;  // bytes per bulk copy instruction (table staging)
 constexpr int kKeyStride = 129;         // second-level keys per first-byte class (two-level sort)
@@ -135,6 +136,7 @@ struct WalkParams {
     const uint32_t* live;
     const int32_t* row_order;  // row-wise walk: rows in the order they are handed out, or null
     const int32_t* win_order;  // bucket walk: windows in the order they are handed out, or null
+    int32_t chunk;             // dense walk: states per warp task (kChunk or kSmallChunk)
     // outputs
     uint32_t* mask;
     void* next;

@@ -74,7 +74,10 @@ __device__ __forceinline__ void walk_task_raw(const WalkParams& p, int q0, int n
     }
 }
 
-template <typename TabT, typename OutT, bool HAS_OUT>
+// CHUNK: states per warp task.  kChunk as a rule; kSmallChunk for a build so small that the
+// device's warps would not get two tasks each (a task walks its states one after the other,
+// so its length is latency).  kSmallChunk divides kChunk: tiles still start on a chunk.
+template <typename TabT, typename OutT, bool HAS_OUT, int CHUNK>
 __global__ void __launch_bounds__(kWalkThreads, 1) walk(const WalkParams p) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     __shared__ uint64_t bar;
@@ -127,13 +130,13 @@ __global__ void __launch_bounds__(kWalkThreads, 1) walk(const WalkParams p) {
                 return;
             }
         }
-        const int nchunks = (w_rows + kChunk - 1) / kChunk;
+        const int nchunks = (w_rows + CHUNK - 1) / CHUNK;
         const int64_t ntasks = static_cast<int64_t>(nchunks) * p.G;
         for (int64_t t = wg; t < ntasks; t += TW) {
             const int chunk = static_cast<int>(t / p.G);
             const int g = static_cast<int>(t - static_cast<int64_t>(chunk) * p.G);
-            const int q0 = w_q0 + chunk * kChunk;
-            const int nq = min(kChunk, w_q0 + w_rows - q0);
+            const int q0 = w_q0 + chunk * CHUNK;
+            const int nq = min(CHUNK, w_q0 + w_rows - q0);
             if (raw) {
                 walk_task_raw<OutT, HAS_OUT>(p, q0, nq, g, lane);
             } else {
@@ -157,7 +160,8 @@ __global__ void __launch_bounds__(kWalkThreads, 1) walk(const WalkParams p) {
 
 template <typename TabT, typename OutT, bool HAS_OUT>
 cudaError_t launch_walk(const WalkParams& p, int grid, cudaStream_t stream) {
-    auto kernel = walk<TabT, OutT, HAS_OUT>;
+    auto kernel = p.chunk == kSmallChunk ? walk<TabT, OutT, HAS_OUT, kSmallChunk>
+                                         : walk<TabT, OutT, HAS_OUT, kChunk>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(p.smem_cap));
     if (e != cudaSuccess) return e;
