@@ -4,8 +4,8 @@ import numpy as np
 import pytest
 import torch
 
-from fsm_inputs import (compile_regex, make_config, paper_float_example_dfa, random_class_dfa,
-                        vocab_from_strings)
+from fsm_inputs import (bpe_like_vocab, compile_regex, make_config, paper_float_example_dfa,
+                        random_class_dfa, vocab_from_strings)
 from oracle import fsm_oracle
 
 pytestmark = pytest.mark.gpu
@@ -122,6 +122,14 @@ def test_state_that_reads_everything_over_a_large_vocabulary():
     mask, nxt = check_index(trans, accept, w.vocab_bytes, w.vocab_offsets, 2, w.eos_id)
     lens = np.diff(w.vocab_offsets)
     assert int(np.unpackbits(mask[0].view(np.uint8)).sum()) == int((lens > 0).sum()) + 1
+
+
+def test_vocabulary_beyond_the_window_ranking():
+    """540,000 tokens are more windows of 32 sorted tokens than the bucket walk ranks in
+    shared memory (it then takes them in index order); the other walks see a long row."""
+    d, _ = random_class_dfa(21, n_live=40, n_classes=30, live_classes_per_state=8)
+    vb, vo = bpe_like_vocab(11, 540_000, zero_length_ids=(539_999,))
+    check_index(d.trans, d.accept, vb, vo, d.dead, 539_999)
 
 
 def test_more_than_127_byte_classes_uses_one_level_buckets():
