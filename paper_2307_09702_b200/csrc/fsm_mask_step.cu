@@ -534,11 +534,13 @@ int step_impl(const void* logits_in, void* logits_out, int32_t logits_dtype, int
         while (k < 8 && static_cast<int64_t>(B) * k < ctas_wanted &&
                vectors / (2 * k * kStepThreads) >= 2)
             k *= 2;
-        // A grid of between one and two and a half waves ends with a thin last wave: halve the
-        // CTAs until there are more waves (B = 1,024: 96 -> 90 us greedy, 155 -> 137 us drawn).
+        // A grid of between one and two and a half waves ends with a thin last wave, which
+        // costs the more the longer a CTA runs: CTAs of twelve or more vectors per thread
+        // are halved until there are more waves (B = 1,024: 96 -> 90 us greedy, 155 -> 137 us
+        // drawn).
         const int64_t places = static_cast<int64_t>(dev.sm_count) * (sample ? 4 : 5);  // resident CTAs
         while (k < 8 && static_cast<int64_t>(B) * k > places &&
-               2 * static_cast<int64_t>(B) * k < 5 * places && vectors / (2 * k * kStepThreads) >= 2)
+               2 * static_cast<int64_t>(B) * k < 5 * places && vectors / (k * kStepThreads) >= 12)
             k *= 2;
     }
 
