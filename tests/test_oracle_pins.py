@@ -11,7 +11,7 @@ import pytest
 from fsm_inputs import (compile_regex, f32_to_bf16_bits, make_config, paper_float_example_dfa,
                         paper_name_dfa, random_class_dfa, signed_decimal_dfa, token_bytes,
                         vocab_from_strings)
-from oracle import alg34_literal, fsm_oracle
+from oracle import fsm_oracle, token_major
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -64,7 +64,7 @@ def test_paper_name_example_sequences():
             accepting = {int(x) for x in f[1:]}
     dfa = paper_name_dfa()
     assert {q for q in range(dfa.Q) if dfa.accept[q]} == accepting
-    assert alg34_literal.find_sub_sequences(dfa.trans, dfa.dead, b"f") == want
+    assert token_major.state_sequences(dfa.trans, dfa.dead, b"f") == want
     vb, vo = vocab_from_strings(["f"])
     mask, nxt, _ = fsm_oracle.index_build(dfa.trans, dfa.accept, vb, vo, dfa.dead)
     for z in want:
@@ -83,7 +83,7 @@ def test_token_major_algorithms_agree_with_state_major_definition(seed):
     vocab[13] = b""
     vb, vo = vocab_from_strings(vocab)
     mask, nxt, _ = fsm_oracle.index_build(dfa.trans, dfa.accept, vb, vo, dfa.dead)
-    sigma, end = alg34_literal.map_states_to_vocab(dfa.trans, dfa.dead, vocab)
+    sigma, end = token_major.index_by_token(dfa.trans, dfa.dead, vocab)
     for q in range(dfa.Q):
         assert allowed_set(mask, q, len(vocab)) == sigma[q]
         for v in range(len(vocab)):
@@ -317,6 +317,36 @@ def test_mask_step_against_numpy(dtype):
     st2, fin2 = states.copy(), finished.copy()
     tokens2, out2 = fsm_oracle.mask_step(logits, st2, fin2, mask, nxt, dead, eos, write_logits=False)
     assert out2 is None and (tokens2 == tokens).all() and (st2 == st).all() and (fin2 == fin).all()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_mask_step_orders_subnormals_like_numpy(dtype):
+    """Subnormal logits, signed zeros and the smallest normal number are ordered as IEEE
+    floats (NumPy's argmax on the widened values is the definition written out)."""
+    rng = np.random.default_rng(23)
+    N, Q = 400, 2
+    mask = rng.integers(0, 2**32, size=(Q, (N + 31) // 32), dtype=np.uint32)
+    mask[:, -1] &= np.uint32((1 << (N % 32)) - 1)
+    mask[1] = 0
+    nxt = np.zeros((Q, N), dtype=np.int32)
+    if dtype == "bf16":
+        pos = np.array([0x0001, 0x0003, 0x007F, 0x0080, 0x0081, 0x0000], dtype=np.uint16)
+        vals = np.concatenate([pos, pos | np.uint16(0x8000)])
+        widen = lambda a: (a.astype(np.uint32) << 16).view(np.float32)
+    else:
+        pos = np.array([1, 0x12345, 0x7FFFFF, 0x800000, 0x800001, 0], dtype=np.uint32)
+        vals = np.concatenate([pos, pos | np.uint32(0x80000000)]).view(np.float32)
+        widen = lambda a: a
+    bits = np.unpackbits(mask.view(np.uint8), axis=1, bitorder="little")[:, :N].astype(bool)
+    for trial in range(40):
+        top = 1 + trial % len(pos)             # restrict the value set so that every level wins
+        pool = np.concatenate([vals[:top], vals[len(pos):]])
+        logits = rng.choice(pool, size=(1, N))
+        st, fin = np.zeros(1, np.int32), np.zeros(1, np.uint8)
+        tokens, out = fsm_oracle.mask_step(logits, st, fin, mask, nxt, Q - 1, -1)
+        _, tok = np_mask_step_row(widen(logits[0]), bits[0])
+        assert tokens[0] == tok
+        assert widen(logits[0])[tok] == widen(logits[0])[bits[0]].max()
 
 
 def test_mask_step_all_allowed_logits_minus_inf_picks_lowest_allowed_id():
