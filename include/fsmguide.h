@@ -259,14 +259,17 @@ int guided_sample_step(const void* logits_in, void* logits_out, int32_t logits_d
  * (sample == 0) or guided_sample_step (sample != 0; inv_temperature, seed and draw as
  * there), except that the next state of the chosen token is found by binary search among
  * the row's tokens instead of in a dense table.  Same masking, selection and bookkeeping,
- * same results.  A chosen token whose entry is missing (index built with too small a
- * capacity, FSM_FLAG_CSR_OVERFLOW) sends the row to the dead state.
+ * same results.  `capacity` is the number of entries csr_tokens and csr_next hold, as given
+ * to fsm_index_build_csr: nothing beyond it is read.  A chosen token whose entry is missing
+ * (index built with too small a capacity, FSM_FLAG_CSR_OVERFLOW) sends the row to the dead
+ * state.
  */
 int guided_step_csr(const void* logits_in, void* logits_out, int32_t logits_dtype,
                     int64_t row_stride, int32_t* states, uint8_t* finished, int32_t* tokens_out,
                     const uint32_t* allowed_mask, const int64_t* row_offsets,
-                    const int32_t* csr_tokens, const int32_t* csr_next, int32_t Q, int32_t N,
-                    int32_t B, int32_t dead_state, int32_t eos_id, int32_t sample,
+                    const int32_t* csr_tokens, const int32_t* csr_next, int64_t capacity,
+                    int32_t Q, int32_t N, int32_t B, int32_t dead_state, int32_t eos_id,
+                    int32_t sample,
                     float inv_temperature, uint64_t seed, uint64_t draw, int32_t* status_word,
                     void* cuda_stream);
 

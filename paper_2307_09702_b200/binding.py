@@ -72,8 +72,9 @@ def lib() -> ctypes.CDLL:
         L.fsm_index_build_csr.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, vp, vp, i64,
                                           vp, sz, vp, vp]
         L.fsm_index_build_csr.restype = ctypes.c_int
-        L.guided_step_csr.argtypes = [vp, vp, i32, i64, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32,
-                                      i32, i32, ctypes.c_float, ctypes.c_uint64, ctypes.c_uint64, vp, vp]
+        L.guided_step_csr.argtypes = [vp, vp, i32, i64, vp, vp, vp, vp, vp, vp, vp, i64, i32, i32, i32,
+                                      i32, i32, i32, ctypes.c_float, ctypes.c_uint64, ctypes.c_uint64,
+                                      vp, vp]
         L.guided_step_csr.restype = ctypes.c_int
         _lib = L
     return _lib
@@ -180,12 +181,12 @@ def fsm_index_build_csr(dfa_trans, accept, vocab_bytes, vocab_offsets, vocab_nby
 
 
 def guided_step_csr(logits_in, logits_out, logits_dtype, row_stride, states, finished, tokens_out,
-                    allowed_mask, row_offsets, csr_tokens, csr_next, Q, N, B, dead_state, eos_id,
-                    sample=0, inv_temperature=1.0, seed=0, draw=0, status_word=None, stream=None) -> int:
+                    allowed_mask, row_offsets, csr_tokens, csr_next, capacity, Q, N, B, dead_state,
+                    eos_id, sample=0, inv_temperature=1.0, seed=0, draw=0, status_word=None, stream=None) -> int:
     return lib().guided_step_csr(_ptr(logits_in), _ptr(logits_out), logits_dtype, row_stride,
                                  _ptr(states), _ptr(finished), _ptr(tokens_out), _ptr(allowed_mask),
-                                 _ptr(row_offsets), _ptr(csr_tokens), _ptr(csr_next), Q, N, B,
-                                 dead_state, eos_id, sample, inv_temperature,
+                                 _ptr(row_offsets), _ptr(csr_tokens), _ptr(csr_next), capacity, Q, N,
+                                 B, dead_state, eos_id, sample, inv_temperature,
                                  seed & 0xFFFFFFFFFFFFFFFF, draw & 0xFFFFFFFFFFFFFFFF,
                                  _ptr(status_word), _stream(stream))
 

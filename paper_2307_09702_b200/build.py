@@ -11,8 +11,12 @@ CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libfsmguide.so")
 SOURCES = ["fsm_api.cu", "fsm_index.cu", "fsm_mask_step.cu"]
+# No --use_fast_math: the decode step compares logits as IEEE floats, subnormals included
+# (that flag flushes them to zero), and nothing on the path needs approximate division or
+# transcendentals.
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "--use_fast_math", "-Xcompiler", "-fPIC"]
+              "-ftz=false", "-prec-div=true", "-prec-sqrt=true", "-fmad=true",
+              "-Xcompiler", "-fPIC"]
 
 
 def _nvcc() -> str:

@@ -11,7 +11,7 @@
 //   4. walk            dense: every (state, token) pair walked by warp tiles;
 //      walk_sparse     only tokens of readable buckets walked, rows assembled slice by slice;
 //      mask_onebyte + walk_buckets   bitmask-only builds
-// If verification in 3 fails (a 64-bit hash collision) the walk reads the uncompressed
+// If verification in 2 fails (a 64-bit hash collision) the walk reads the uncompressed
 // table instead, so the result is exact in every case.
 #include "fsm_index_common.cuh"
 #include "fsm_index_dense.cuh"
@@ -32,7 +32,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
                     int32_t dead_state, int32_t eos_id, int32_t q_begin, int32_t q_end,
                     uint32_t* allowed_mask, void* next_state, int32_t state_dtype, void* workspace,
                     size_t workspace_bytes, int32_t* status_word, void* cuda_stream,
-                    bool dense_only) {
+                    bool dense_only, bool want_tok_head = false) {
     using namespace fsm;
     if (Q <= 0 || N <= 0 || vocab_nbytes < 0 || N > 0x7FFFFFE0) return FSM_ERR_SHAPE;
     if (!dfa_trans || !accept || !vocab_offsets || !allowed_mask) return FSM_ERR_NULL;
@@ -71,12 +71,15 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
         tune.walk_algo == 2 || (tune.walk_algo == 0 && q_end - q_begin >= dev.sm_count);
     // Bitmask-only builds take the bucket walk (no dense rows to assemble).
     // (like the row-wise walk it needs enough rows to fill the device)
-    const bool bucket = next_state == nullptr && !dense_only &&
+    // Both work-avoiding walks need a vocabulary their slice counters and shared memory hold;
+    // a larger one takes the dense walk.
+    const bool sparse_fits =
+        !dense_only && (N + 255) / 256 <= kMaxSlices &&
+        sparse_table_offset<int32_t>(N) + 4096 <= static_cast<size_t>(dev.smem_optin - 2048);
+    const bool bucket = next_state == nullptr && sparse_fits &&
                         (tune.walk_algo == 3 ||
                          (tune.walk_algo == 0 && q_end - q_begin >= dev.sm_count));
-    const bool sparse = (bucket || want_sparse) && !dense_only &&
-                        (N + 255) / 256 <= kMaxSlices &&
-                        sparse_table_offset<int32_t>(N) + 4096 <= static_cast<size_t>(dev.smem_optin - 2048);
+    const bool sparse = (bucket || want_sparse) && sparse_fits;
 
     const int hash_blocks = Q < kHashBlocks ? Q : kHashBlocks;
     if (launch_overlapped(hash_columns, dim3(hash_blocks), dim3(256 * kHashRowLanes), 0, stream,
@@ -106,7 +109,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
                               vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
                               ws.partial, hash_blocks, ws.meta, ws.cls, static_cast<int32_t*>(ws.table),
                               tok_cls, ws.tok_len, live, count2, planes,
-                              bucket ? ws.tok_head : nullptr, status_word) != cudaSuccess)
+                              want_tok_head ? ws.tok_head : nullptr, status_word) != cudaSuccess)
             return FSM_ERR_CUDA;
     } else {
         auto k = prepare_all<uint16_t>;
@@ -117,7 +120,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
                               vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
                               ws.partial, hash_blocks, ws.meta, ws.cls, static_cast<uint16_t*>(ws.table),
                               tok_cls, ws.tok_len, live, count2, planes,
-                              bucket ? ws.tok_head : nullptr, status_word) != cudaSuccess)
+                              want_tok_head ? ws.tok_head : nullptr, status_word) != cudaSuccess)
             return FSM_ERR_CUDA;
     }
     if (sparse) {
@@ -298,7 +301,8 @@ extern "C" int fsm_index_build_csr(const int32_t* dfa_trans, const uint8_t* acce
     const int rc = build_rows_impl(dfa_trans, accept, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N,
                                    dead_state, eos_id, 0, Q, allowed_mask, dense_next,
                                    dense_next ? FSM_STATE_U16 : FSM_STATE_I32, workspace,
-                                   workspace_bytes, status_word, cuda_stream, false);
+                                   workspace_bytes, status_word, cuda_stream, false,
+                                   /*want_tok_head=*/dense_next == nullptr);
     if (rc != FSM_OK) return rc;
     const DeviceInfo& dev = device_info();
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

@@ -200,7 +200,10 @@ csr_fill(const WalkParams p, const uint16_t* __restrict__ tok_head,
                     }
                 }
                 const uint32_t m = __ballot_sync(kFullWarp, walk);
-                if (nlong + __popc(m) > kLongCap) walk_longs();
+                if (nlong + __popc(m) > kLongCap) {
+                    __syncwarp();  // the entries other lanes set aside are visible to the walk
+                    walk_longs();
+                }
                 if (walk) longs[nlong + __popc(m & ((1u << lane) - 1u))] = make_int2(at + j, v);
                 nlong += __popc(m);
             }

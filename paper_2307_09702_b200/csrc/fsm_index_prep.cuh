@@ -212,6 +212,7 @@ prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab
              v += static_cast<int64_t>(gridDim.x) * kPrepTokens) {
             uint32_t w[4] = {static_cast<uint32_t>(C), 0, 0, 0};  // an empty token reads the null class
             int len = 0;
+            uint32_t first_byte = 0;
             if (v < N && v != eos_id) {
                 const int64_t o0 = vocab_offsets[v], o1 = vocab_offsets[v + 1];
                 if (o0 < 0 || o1 < o0 || o1 > vocab_nbytes) {
@@ -224,6 +225,7 @@ prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab
 #pragma unroll
                     for (int i = 0; i < kInlineBytes; ++i)  // independent loads, issued together
                         raw[i] = i < n ? vocab_bytes[o0 + i] : 0;
+                    first_byte = raw[0];
 #pragma unroll
                     for (int i = 0; i < kInlineBytes; ++i)
                         if (i < n) w[i >> 2] |= static_cast<uint32_t>(s_cls[raw[i]]) << ((i & 3) * 8);
@@ -231,6 +233,8 @@ prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab
             }
             tok_cls[v] = make_uint4(w[0], w[1], w[2], w[3]);
             tok_len[v] = static_cast<uint8_t>(len);
+            if (tok_head != nullptr && v < N)  // first byte and length, for the compressed rows
+                tok_head[v] = static_cast<uint16_t>(first_byte | (static_cast<uint32_t>(len) << 8));
         }
     }
     // ---- bucket keys of the tokens, kPrepTokens at a time

@@ -22,7 +22,7 @@
 //             memory only sees full, write-once traffic for the outputs: the tokens
 //             whose first byte q cannot read cost no lookup at all.
 //
-// Three CTA barriers per row.  Results are identical to the dense walk.
+// Two CTA barriers per row.  Results are identical to the dense walk.
 #pragma once
 
 #include "fsm_index_common.cuh"

@@ -38,6 +38,7 @@ struct StepParams {
     const int64_t* csr_offsets;
     const int32_t* csr_tokens;
     const int32_t* csr_next;
+    int64_t csr_capacity;  // entries the two arrays hold
     // sampling
     float inv_temperature;
     uint32_t seed_lo, seed_hi, draw_lo, draw_hi;
@@ -129,7 +130,8 @@ __device__ __forceinline__ int locate(const uint32_t (&w)[NW], uint32_t bits, fl
 // logit / temperature + G with G a standard Gumbel variate.  The random bits come from
 // Philox4x32-10 (Salmon et al., SC'11) with key = seed and counter = (token id / 4, batch
 // row, draw number); token v uses output word v % 4.  Every floating-point step is an
-// explicitly rounded fp32 operation, so the result does not depend on compiler flags.
+// explicitly rounded fp32 operation and the library is built without flush-to-zero, so
+// subnormal logits take part in the score as they are.
 __device__ __forceinline__ uint32_t philox_word(uint32_t v, uint32_t row, const StepParams& p) {
     uint32_t c0 = v >> 2, c1 = row, c2 = p.draw_lo, c3 = p.draw_hi;
     uint32_t k0 = p.seed_lo, k1 = p.seed_hi;
@@ -308,8 +310,8 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
         // Per thread and pass: the bitmask bits of kGroup vectors are fetched first (one
         // round trip to L2), then the vectors are streamed kUnroll at a time - every needed
         // logits load of a batch is issued before any arithmetic.  Two loads in flight per
-        // thread keep the kernel at 64 registers (four CTAs per SM), which measured faster
-        // than four or eight loads at 80 to 160 registers.
+        // thread keep the greedy kernel at 48 registers (five CTAs per SM), which measured
+        // faster than four or eight loads at 80 to 160 registers.
         constexpr int kUnroll = 2, kGroup = 4;
         const int nvec = p.N / EPV;
         constexpr uint32_t kBitsMask = (EPV == 32) ? 0xFFFFFFFFu : ((1u << EPV) - 1u);
@@ -448,8 +450,13 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
         } else {
             p.tokens[row] = b.idx;
             if (p.csr_offsets != nullptr) {
-                // the row's tokens are in increasing order: binary search for the chosen one
-                int64_t lo = p.csr_offsets[q], hi = p.csr_offsets[q + 1];
+                // the row's tokens are in increasing order: binary search for the chosen one.
+                // row_offsets is complete even when the index has more entries than the arrays
+                // hold, so the search stays inside the part that exists.
+                const int64_t cap = p.csr_capacity;
+                int64_t lo = min(max(p.csr_offsets[q], static_cast<int64_t>(0)), cap);
+                const int64_t end = min(max(p.csr_offsets[q + 1], lo), cap);
+                int64_t hi = end;
                 while (lo < hi) {
                     const int64_t mid = (lo + hi) >> 1;
                     if (p.csr_tokens[mid] < b.idx)
@@ -457,7 +464,7 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
                     else
                         hi = mid;
                 }
-                const bool found = lo < p.csr_offsets[q + 1] && p.csr_tokens[lo] == b.idx;
+                const bool found = lo < end && p.csr_tokens[lo] == b.idx;
                 p.states[row] = found ? p.csr_next[lo] : p.dead;  // (an entry lost to a too small
                                                                   // capacity leads to dead)
             } else {
@@ -496,11 +503,13 @@ int step_impl(const void* logits_in, void* logits_out, int32_t logits_dtype, int
               int32_t N, int32_t B, int32_t dead_state, int32_t eos_id, bool sample,
               float inv_temperature, uint64_t seed, uint64_t draw, int32_t* status_word,
               void* cuda_stream, const int64_t* csr_offsets = nullptr,
-              const int32_t* csr_tokens = nullptr, const int32_t* csr_next = nullptr) {
+              const int32_t* csr_tokens = nullptr, const int32_t* csr_next = nullptr,
+              int64_t csr_capacity = 0) {
     using namespace fsm;
     if (Q <= 0 || N <= 0 || B < 0 || row_stride < N) return FSM_ERR_SHAPE;
     if (!logits_in || !states || !finished || !tokens_out || !allowed_mask) return FSM_ERR_NULL;
-    if (csr_offsets ? (!csr_tokens || !csr_next) : !next_state) return FSM_ERR_NULL;
+    if (csr_offsets ? (csr_capacity > 0 && (!csr_tokens || !csr_next)) : !next_state) return FSM_ERR_NULL;
+    if (csr_capacity < 0) return FSM_ERR_SHAPE;
     if (logits_dtype != FSM_LOGITS_F32 && logits_dtype != FSM_LOGITS_BF16) return FSM_ERR_DTYPE;
     if (state_dtype != FSM_STATE_I32 && state_dtype != FSM_STATE_U16) return FSM_ERR_DTYPE;
     if (state_dtype == FSM_STATE_U16 && Q > 65535) return FSM_ERR_DTYPE;
@@ -565,6 +574,7 @@ int step_impl(const void* logits_in, void* logits_out, int32_t logits_dtype, int
     p.csr_offsets = csr_offsets;
     p.csr_tokens = csr_tokens;
     p.csr_next = csr_next;
+    p.csr_capacity = csr_capacity;
     p.inv_temperature = inv_temperature;
     p.seed_lo = static_cast<uint32_t>(seed);
     p.seed_hi = static_cast<uint32_t>(seed >> 32);
@@ -615,8 +625,8 @@ extern "C" int guided_step_csr(const void* logits_in, void* logits_out, int32_t 
                                int64_t row_stride, int32_t* states, uint8_t* finished,
                                int32_t* tokens_out, const uint32_t* allowed_mask,
                                const int64_t* row_offsets, const int32_t* csr_tokens,
-                               const int32_t* csr_next, int32_t Q, int32_t N, int32_t B,
-                               int32_t dead_state, int32_t eos_id, int32_t sample,
+                               const int32_t* csr_next, int64_t capacity, int32_t Q, int32_t N,
+                               int32_t B, int32_t dead_state, int32_t eos_id, int32_t sample,
                                float inv_temperature, uint64_t seed, uint64_t draw,
                                int32_t* status_word, void* cuda_stream) {
     if (!row_offsets) return FSM_ERR_NULL;
@@ -627,5 +637,5 @@ extern "C" int guided_step_csr(const void* logits_in, void* logits_out, int32_t 
     return step_impl(logits_in, logits_out, logits_dtype, row_stride, states, finished, tokens_out,
                      allowed_mask, nullptr, FSM_STATE_I32, Q, N, B, dead_state, eos_id, sample != 0,
                      sample ? inv_temperature : 1.0f, seed, draw, status_word, cuda_stream,
-                     row_offsets, csr_tokens, csr_next);
+                     row_offsets, csr_tokens, csr_next, capacity);
 }

@@ -117,10 +117,74 @@ def test_decode_steps_on_compressed_rows_match_the_oracle(sample):
                                                 threads=THREADS)
         dx = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
         rc = fg.guided_step_csr(dx, dx, fg.FSM_LOGITS_BF16, w.N, d_st, d_fin, d_tok, mask, off, tok, nxt,
-                                d.Q, w.N, B, d.dead, w.eos_id, sample, 10.0, 77, step, status)
+                                tok.numel(), d.Q, w.N, B, d.dead, w.eos_id, sample, 10.0, 77, step,
+                                status)
         assert rc == 0
         torch.cuda.synchronize()
         assert (d_tok.cpu().numpy() == tok_o).all()
         assert (d_st.cpu().numpy() == st_o).all() and (d_fin.cpu().numpy() == fin_o).all()
         assert (dx.view(torch.int16).cpu().numpy().view(np.uint16) == out_o).all()
     assert int(status.item()) == 0
+
+
+def test_decode_step_on_an_overflowed_index_stays_inside_the_arrays():
+    """An index built with half the capacity it needs: row_offsets is complete, the entry
+    arrays end at `capacity`.  The step must not look beyond them (the words behind are
+    canaries that would send a row to a wrong state): a chosen token whose entry exists
+    advances as usual, one whose entry is missing goes to the dead state."""
+    w = make_config(2)
+    d = w.dfa
+    o_mask, want_off, want_tok, want_next = fsm_oracle.index_csr(
+        d.trans, d.accept, w.vocab_bytes, w.vocab_offsets, d.dead, w.eos_id, threads=THREADS)
+    total = int(want_off[-1])
+    cap = total // 2
+    mask, off, tok, nxt, status = build_csr(d.trans, d.accept, w.vocab_bytes, w.vocab_offsets, d.dead,
+                                            w.eos_id, cap)
+    assert status == 32
+    # entry arrays followed by canaries: every token id, each "leading" to state 1
+    canary_tok = torch.arange(w.N, dtype=torch.int32, device="cuda").repeat(4)
+    tok_c = torch.cat([tok[:cap], canary_tok])
+    nxt_c = torch.cat([nxt[:cap], torch.ones_like(canary_tok)])
+    live = [q for q in range(d.Q) if want_off[q + 1] > want_off[q]]
+    B = len(live)
+    states = np.array(live, dtype=np.int32)
+    d_st = torch.from_numpy(states.copy()).cuda()
+    d_fin = torch.zeros(B, dtype=torch.uint8, device="cuda")
+    d_tok = torch.zeros(B, dtype=torch.int32, device="cuda")
+    st_word = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((B, w.N)).astype(np.float32)
+    dx = torch.from_numpy(x).cuda()
+    rc = fg.guided_step_csr(dx, None, fg.FSM_LOGITS_F32, w.N, d_st, d_fin, d_tok, mask, off, tok_c,
+                            nxt_c, cap, d.Q, w.N, B, d.dead, w.eos_id, 0, 1.0, 0, 0, st_word)
+    assert rc == 0
+    torch.cuda.synchronize()
+    got_tok, got_st = d_tok.cpu().numpy(), d_st.cpu().numpy()
+    n_missing = 0
+    for i, q in enumerate(live):
+        lo, hi = int(want_off[q]), int(want_off[q + 1])
+        row_tok = want_tok[lo:hi]
+        choice = int(row_tok[np.argmax(x[i, row_tok])])        # allowed token with the largest logit
+        assert got_tok[i] == choice
+        if choice == w.eos_id:
+            continue
+        at = lo + int(np.searchsorted(row_tok, choice))
+        if at < cap:
+            assert got_st[i] == want_next[at]
+        else:
+            n_missing += 1
+            assert got_st[i] == d.dead
+    assert n_missing > 0
+
+
+@pytest.mark.parametrize("algo", [1, 2])
+def test_compressed_rows_under_every_walk_algorithm(algo):
+    """300 states: the rows are cut out of the bitmask (no dense table in the workspace),
+    whichever walk built it."""
+    d, _ = random_class_dfa(300, n_live=300, n_classes=40, live_classes_per_state=9)
+    vb, vo = bpe_like_vocab(7, 5000, zero_length_ids=(4999,))
+    fg.fsm_debug_set(6, algo)
+    try:
+        check_csr(d.trans, d.accept, vb, vo, d.dead, 4999)
+    finally:
+        fg.fsm_debug_set(6, 0)

@@ -34,8 +34,9 @@ def random_index(rng, Q, N, allowed_frac=0.25):
 
 
 def run_case(rng, Q, N, B, dtype, mode, k=0, stride_pad=0, state_dtype=0, eos=5, coarse=True,
-             sample=None):
-    """``sample`` = (inv_temperature, seed, draw) runs the categorical draw instead of argmax."""
+             sample=None, special=None):
+    """``sample`` = (inv_temperature, seed, draw) runs the categorical draw instead of argmax;
+    ``special(x, mask, states)`` may rewrite the fp32 logits before they are converted."""
     mask, nxt = random_index(rng, Q, N)
     mask[3] = 0
     x = rng.standard_normal((B, N)).astype(np.float32) * 2
@@ -52,6 +53,8 @@ def run_case(rng, Q, N, B, dtype, mode, k=0, stride_pad=0, state_dtype=0, eos=5,
     if B > 6 and eos >= 0:
         mask[states[6], eos >> 5] |= np.uint32(1 << (eos & 31))
         x[6, eos] = 1000.0
+    if special is not None:
+        special(x, mask, states)
     host_logits = f32_to_bf16_bits(x) if dtype == "bf16" else x
     st_o, fin_o = states.copy(), finished.copy()
     if sample is None:
@@ -200,6 +203,91 @@ def test_sample_workload_5_shape_steps_match_oracle():
         assert (d_tok.cpu().numpy() == tok_o).all()
         assert (d_st.cpu().numpy() == st_o).all() and (d_fin.cpu().numpy() == fin_o).all()
         assert (x.view(torch.int16).cpu().numpy().view(np.uint16) == out_o).all()
+
+
+def _tiny_values(dtype):
+    """Positive values below, at and just above the subnormal boundary, exactly
+    representable in ``dtype`` (bf16 keeps 8 significant bits of the fp32 pattern)."""
+    if dtype == "bf16":
+        bits = [0x00010000, 0x00030000, 0x007F0000, 0x00800000, 0x00810000]
+    else:
+        bits = [0x00000001, 0x00012345, 0x007FFFFF, 0x00800000, 0x00800001]
+    return np.array(bits, dtype=np.uint32).view(np.float32)
+
+
+def _subnormal_rows(dtype):
+    """Rewrites rows 0, 5, 7 and 8 so that the comparison among the allowed logits is decided
+    by subnormals, signed zeros and the smallest normal number, with ties among them; a
+    comparison that flushed subnormals to zero would pick other tokens."""
+    tiny = _tiny_values(dtype)
+
+    def special(x, mask, states):
+        B, N = x.shape
+        rng = np.random.default_rng(B * 31 + N)
+
+        def allowed_ids(row):
+            q = states[row]
+            bits = np.unpackbits(mask[q].view(np.uint8), bitorder="little")[:N]
+            ids = np.flatnonzero(bits)
+            assert len(ids) >= 8, "the seeded case gives these rows a non-empty state"
+            return ids
+
+        # row 0: every allowed logit in {-tiny, -0, +0, +tiny}; the largest subnormal appears
+        # several times, zeros sit at lower ids
+        ids = allowed_ids(0)
+        vals = np.concatenate([tiny[:3], -tiny[:3], [0.0, -0.0]]).astype(np.float32)
+        x[0, ids] = rng.choice(vals, size=len(ids))
+        x[0, ids[:2]] = [0.0, -0.0]
+        x[0, ids[len(ids) // 2]] = tiny[2]
+        x[0, ids[-1]] = tiny[2]
+        # row 5: all allowed logits are negative subnormals or -0.0 after some +0.0-free prefix:
+        # the maximum is a signed zero, which must not tie with a flushed subnormal before it
+        ids = allowed_ids(5)
+        x[5, ids] = -rng.choice(tiny[:3], size=len(ids))
+        x[5, ids[len(ids) // 3]] = -0.0
+        x[5, ids[2 * len(ids) // 3]] = 0.0
+        # row 7: smallest normal against the largest subnormal, both repeated
+        ids = allowed_ids(7)
+        x[7, ids] = rng.choice(np.array([tiny[2], -tiny[3], tiny[1], 0.0], dtype=np.float32), size=len(ids))
+        x[7, ids[len(ids) // 2]] = tiny[3]
+        x[7, ids[-2]] = tiny[3]
+        # row 8: smallest subnormal alone above zeros
+        ids = allowed_ids(8)
+        x[8, ids] = rng.choice(np.array([0.0, -0.0, -tiny[0]], dtype=np.float32), size=len(ids))
+        x[8, ids[-3]] = tiny[0]
+    return special
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("N,pad", [(5000, 0), (1003, 5)])
+def test_subnormal_logits_compare_as_ieee_floats(dtype, N, pad):
+    """Greedy selection among subnormals, signed zeros and the smallest normal (wide and
+    narrow row alignment): bit-exact against the oracle."""
+    if dtype == "f32":
+        pad = (-N) % 4 if (N + pad) % 4 else pad
+    else:
+        pad = pad if (N + pad) % 8 == 0 else (-N) % 8
+    for mode in ("inplace", "select"):
+        tok = run_case(np.random.default_rng(3), Q=11, N=N, B=9, dtype=dtype, mode=mode,
+                       stride_pad=pad, special=_subnormal_rows(dtype))
+        assert (tok[[0, 5, 7, 8]] >= 0).all()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("k", [1, 4])
+def test_subnormal_logits_in_the_categorical_draw(dtype, k):
+    """With a huge inverse temperature a subnormal logit moves the score; the product must be
+    formed from the unflushed value."""
+    tiny = _tiny_values(dtype)
+
+    def special(x, mask, states):
+        rng = np.random.default_rng(17)
+        x[:] = rng.choice(np.concatenate([tiny[:3], -tiny[:3], [0.0, -0.0]]).astype(np.float32),
+                          size=x.shape)
+
+    for inv_t in (1.0e38, 3.0e37):
+        run_case(np.random.default_rng(k), Q=11, N=6000, B=9, dtype=dtype, mode="inplace", k=k,
+                 sample=(inv_t, 4242, 9), coarse=False, special=special)
 
 
 def test_u16_next_state_and_smooth_logits():
