@@ -9,14 +9,15 @@
 //                      walk) or bucket key counts (work-avoiding walks)
 //   3. sort_all        work-avoiding walks only: tokens sorted by (first, second) byte class
 //   4. walk            dense: every (state, token) pair walked by warp tiles;
-//      walk_sparse     only tokens of readable buckets walked, rows assembled slice by slice;
+//      walk_rows       rows filled from a per-row table, longer tokens of readable buckets
+//                      walked and patched in;
 //      mask_onebyte + walk_buckets   bitmask-only builds
 // If verification in 2 fails (a 64-bit hash collision) the walk reads the uncompressed
 // table instead, so the result is exact in every case.
 #include "fsm_index_common.cuh"
 #include "fsm_index_dense.cuh"
 #include "fsm_index_prep.cuh"
-#include "fsm_index_sparse.cuh"
+#include "fsm_index_rows.cuh"
 #include "fsm_index_bucket.cuh"
 #include "fsm_index_csr.cuh"
 
@@ -62,24 +63,20 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     Workspace ws = carve(workspace, Q, N);
     const bool wide = Q > 65535;
     const int G = (N + 31) / 32;
-    int cap = dev.smem_optin - 2048;  // static shared memory and alignment slack
+    int cap = dev.smem_optin - kStaticSmemSlack;  // static shared memory and alignment slack
     if (tune.smem_table_cap > 0 && tune.smem_table_cap < cap) cap = tune.smem_table_cap;
-    // The sparse walk needs the survivor scratch and room for its per-warp staging.
-    // Automatic choice: the sparse walk works row by row, one CTA per row at a time, so it
-    // needs at least one row per SM to fill the device; small automata take the dense walk.
-    const bool want_sparse =
-        tune.walk_algo == 2 || (tune.walk_algo == 0 && q_end - q_begin >= dev.sm_count);
-    // Bitmask-only builds take the bucket walk (no dense rows to assemble).
-    // (like the row-wise walk it needs enough rows to fill the device)
-    // Both work-avoiding walks need a vocabulary their slice counters and shared memory hold;
-    // a larger one takes the dense walk.
-    const bool sparse_fits =
-        !dense_only && (N + 255) / 256 <= kMaxSlices &&
-        sparse_table_offset<int32_t>(N) + 4096 <= static_cast<size_t>(dev.smem_optin - 2048);
-    const bool bucket = next_state == nullptr && sparse_fits &&
-                        (tune.walk_algo == 3 ||
-                         (tune.walk_algo == 0 && q_end - q_begin >= dev.sm_count));
-    const bool sparse = (bucket || want_sparse) && sparse_fits;
+    // Automatic choice: the work-avoiding walks work row by row (or window by window) with
+    // one CTA per SM, so they need at least one row per SM to fill the device; small automata
+    // take the dense walk.  With a next-state table: the row-wise fill-and-patch walk;
+    // bitmask-only builds: the bucket walk.
+    const bool enough_rows = q_end - q_begin >= dev.sm_count;
+    const bool rows_fits =
+        !dense_only && rows_min_smem<int32_t>() <= static_cast<size_t>(dev.smem_optin - kStaticSmemSlack);
+    const bool bucket = next_state == nullptr && !dense_only &&
+                        (tune.walk_algo == 3 || (tune.walk_algo == 0 && enough_rows));
+    const bool rows = !bucket && rows_fits &&
+                      (tune.walk_algo == 2 || (tune.walk_algo == 0 && enough_rows));
+    const bool sparse = bucket || rows;  // tokens sorted by bucket key
 
     const int hash_blocks = Q < kHashBlocks ? Q : kHashBlocks;
     if (launch_overlapped(hash_columns, dim3(hash_blocks), dim3(256 * kHashRowLanes), 0, stream,
@@ -97,7 +94,8 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     int32_t* row_order = sparse && !bucket ? ws.row_order : nullptr;
     // (the ranking of the windows counts them in kKeys words of shared memory)
     int32_t* win_order = bucket && sparse && (N + 31) / 32 <= kKeys ? ws.win_order : nullptr;
-    uint32_t* planes = bucket ? ws.planes : nullptr;
+    uint32_t* planes = bucket || rows ? ws.planes : nullptr;
+    uint8_t* tok_c1 = rows ? ws.tok_c1 : nullptr;
     const size_t key_smem = sparse ? kKeys * sizeof(int) : 0;
     const size_t sort_smem = (kKeysPad + kKeys) * sizeof(int);
     if (wide) {
@@ -109,7 +107,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
                               vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
                               ws.partial, hash_blocks, ws.meta, ws.cls, static_cast<int32_t*>(ws.table),
                               tok_cls, ws.tok_len, live, count2, planes,
-                              want_tok_head ? ws.tok_head : nullptr, status_word) != cudaSuccess)
+                              want_tok_head ? ws.tok_head : nullptr, tok_c1, status_word) != cudaSuccess)
             return FSM_ERR_CUDA;
     } else {
         auto k = prepare_all<uint16_t>;
@@ -120,7 +118,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
                               vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
                               ws.partial, hash_blocks, ws.meta, ws.cls, static_cast<uint16_t*>(ws.table),
                               tok_cls, ws.tok_len, live, count2, planes,
-                              want_tok_head ? ws.tok_head : nullptr, status_word) != cudaSuccess)
+                              want_tok_head ? ws.tok_head : nullptr, tok_c1, status_word) != cudaSuccess)
             return FSM_ERR_CUDA;
     }
     if (sparse) {
@@ -131,7 +129,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
         if (launch_overlapped(sort_all, dim3(sort_blocks + (row_order || win_order ? 1 : 0)), dim3(kPrepThreads),
                               sort_smem, stream, vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id,
                               ws.meta, ws.cls, ws.count2, ws.cursor2, ws.start2, ws.gstart, ws.srec,
-                              ws.sid, live, q_begin, q_end, row_order, win_order) != cudaSuccess)
+                              live, q_begin, q_end, row_order, win_order) != cudaSuccess)
             return FSM_ERR_CUDA;
     }
     if (cudaGetLastError() != cudaSuccess) return FSM_ERR_CUDA;
@@ -154,8 +152,8 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     p.tok_cls = ws.tok_cls;
     p.tok_len = ws.tok_len;
     p.srec = ws.srec;
-    p.sid = ws.sid;
     p.planes = ws.planes;
+    p.tok_c1 = ws.tok_c1;
     p.live = ws.live;
     p.row_order = row_order;
     p.chunk = kChunk;
@@ -167,8 +165,8 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     p.mask = allowed_mask;
     p.next = next_state;
     p.status = status_word;
-    const int min_cap = sparse ? static_cast<int>(sparse_table_offset<int32_t>(N)) + 4096
-                               : (kChunk + 4) * kMaxCs * 4;
+    const int min_cap = rows ? static_cast<int>(rows_min_smem<int32_t>())
+                             : (kChunk + 4) * kMaxCs * 4;
     if (cap < min_cap) cap = min_cap;
     p.smem_cap = static_cast<uint32_t>(cap) / 128 * 128;
 
@@ -184,18 +182,17 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
         grid = tasks;  // capped at one CTA per SM below; its warps take the tasks round-robin
     }
     if (grid > dev.sm_count) grid = dev.sm_count;
-    if (sparse && grid > kMaxSparseCtas) grid = kMaxSparseCtas;
     if (tune.walk_ctas > 0 && tune.walk_ctas < grid) grid = tune.walk_ctas;
     const int prof = profile_begin(stream);
     cudaError_t e;
     if (bucket)
         e = wide ? launch_bucket<int32_t>(p, dev.sm_count, stream)
                  : launch_bucket<uint16_t>(p, dev.sm_count, stream);
-    else if (sparse)
-        e = wide ? launch_sparse_for<int32_t>(p, ws.survivors, static_cast<int>(grid), state_dtype,
-                                              next_state != nullptr, stream)
-                 : launch_sparse_for<uint16_t>(p, ws.survivors, static_cast<int>(grid), state_dtype,
-                                               next_state != nullptr, stream);
+    else if (rows)
+        e = wide ? launch_rows_for<int32_t>(p, static_cast<int>(grid), state_dtype,
+                                            next_state != nullptr, stream)
+                 : launch_rows_for<uint16_t>(p, static_cast<int>(grid), state_dtype,
+                                             next_state != nullptr, stream);
     else
         e = wide ? launch_walk_for<int32_t>(p, static_cast<int>(grid), state_dtype,
                                             next_state != nullptr, stream)

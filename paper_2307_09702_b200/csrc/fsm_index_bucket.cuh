@@ -18,7 +18,7 @@
 #pragma once
 
 #include "fsm_index_common.cuh"
-#include "fsm_index_sparse.cuh"
+#include "fsm_index_rows.cuh"
 
 namespace fsm {
 namespace {
@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(kObThreads) mask_onebyte(const WalkParams p) {
     const int c_smem = min(C, kObSmemClasses);
     for (int i = threadIdx.x; i < c_smem * kObWords; i += kObThreads) {
         const int wd = w0 + (i & (kObWords - 1));
-        s_pl[i] = wd < p.G ? p.planes[static_cast<size_t>(i / kObWords) * p.G + wd] : 0;
+        s_pl[i] = wd < p.G ? p.planes[static_cast<size_t>(i / kObWords) * plane_stride(p.G) + wd] : 0;
     }
     __syncthreads();
     const int eos_word = p.eos_id >= 0 ? (p.eos_id >> 5) - w0 : -1;
@@ -104,7 +104,7 @@ __global__ void __launch_bounds__(kObThreads) mask_onebyte(const WalkParams p) {
             if (c < kObSmemClasses) {
                 v = *reinterpret_cast<const uint4*>(s_pl + c * kObWords + 4 * lane);
             } else {
-                const uint32_t* pl = p.planes + static_cast<size_t>(c) * p.G + wl;
+                const uint32_t* pl = p.planes + static_cast<size_t>(c) * plane_stride(p.G) + wl;
                 v.x = wl < p.G ? __ldg(pl) : 0u;
                 v.y = wl + 1 < p.G ? __ldg(pl + 1) : 0u;
                 v.z = wl + 2 < p.G ? __ldg(pl + 2) : 0u;
@@ -170,7 +170,7 @@ __device__ __forceinline__ void bucket_tasks(const WalkParams& p, const TabT* __
         int32_t id = -1;
         if (pos < n_sorted) {
             rec = __ldg(p.srec + pos);
-            id = __ldg(p.sid + pos);
+            id = static_cast<int32_t>(rec.w);
         }
         const int len = rec.x & 0xFFu;
         const bool active = id >= 0 && len >= 2;
@@ -200,9 +200,9 @@ __device__ __forceinline__ void bucket_tasks(const WalkParams& p, const TabT* __
                     m &= m - 1;
                     const uint32_t s = __shfl_sync(kFullWarp, s2, l);
                     bool go = same && len > 2;
-                    uint32_t st = walk_rest<TabT, FULL, 2>(tab, Cs, dead, rec, len, s, go);
-                    if (go)  // longer than the inline record and still alive
-                        st = raw_walk(p, st, p.vocab_offsets[id], p.vocab_offsets[id + 1], kInlineBytes);
+                    uint32_t st = walk_rest<TabT, FULL, 2, kSortedInline>(tab, Cs, dead, rec, len, s, go);
+                    if (go)  // longer than the record covers and still alive
+                        st = raw_walk(p, st, p.vocab_offsets[id], p.vocab_offsets[id + 1], kSortedInline);
                     if (same && st != dead)
                         atomicOr(p.mask + static_cast<size_t>(rbase + l) * p.G + word, bit);
                 }

@@ -12,13 +12,14 @@ constexpr int kWalkThreads = 1024;
 constexpr int kWalkWarps = kWalkThreads / 32;
 constexpr int kChunk = 32;              // states per warp task (dense walk)
 constexpr int kSmallChunk = 8;          // the same for builds of few tasks
-constexpr int kInlineBytes = 16;        // token bytes kept in a 16-byte record
+constexpr int kInlineBytes = 16;        // token bytes kept in a 16-byte record (dense walk)
+constexpr int kSortedInline = 12;       // token bytes covered by a sorted record (its last word is the id)
 constexpr uint32_t kBulkChunk = 32768;  // bytes per bulk copy instruction (table staging)
 constexpr int kKeyStride = 129;         // second-level keys per first-byte class (two-level sort)
 constexpr int kKeys = kKeyStride * kKeyStride;
 constexpr int kTwoLevelMaxC = 127;      // more classes than this: one-level buckets only
 constexpr int kCsrDenseRows = 256;      // smaller automata: compressed rows cut out of a dense table
-constexpr int kMaxSparseCtas = 160;     // CTAs of the sparse walk (one survivor scratch each)
+constexpr int kStaticSmemSlack = 3072;   // static shared memory of the walk kernels, with margin
 
 struct IndexMeta {
     int32_t C;          // number of byte classes (the null class has id C)
@@ -32,20 +33,19 @@ struct Workspace {
     uint8_t* cls;        // [256] byte -> class
     uint64_t* partial;   // [kHashBlocks][256] column hash partial sums
     void* table;         // [Q][Cs] of TabT
-    // dense walk: token records in token order (aliases the sparse walk's arrays)
+    // dense walk: token records in token order (aliases the sorted records)
     uint4* tok_cls;      // [G*32] first 16 class ids of each token
     uint8_t* tok_len;    // [G*32] min(length, 17)
-    // sparse walk: tokens sorted by bucket key
-    uint4* srec;         // [N] {min(len,17), class of byte 1..15}
-    int32_t* sid;        // [N] token id, same order as srec
+    // work-avoiding walks: tokens sorted by bucket key
+    uint4* srec;         // [N] {min(len,13), classes of bytes 1..11, token id}
     int32_t* gstart;     // [257] first sorted position of each first-byte class
-    int32_t* row_ctr;    // [1] rows handed out by the sparse walk beyond the first one per CTA
+    int32_t* row_ctr;    // [1] rows handed out by the row-wise walk beyond the first one per CTA
     int32_t* count2;     // [kKeys] tokens per (first class, second key)
     int32_t* cursor2;    // [kKeys] placement cursors
     int32_t* start2;     // [kKeys] first sorted position of each (first class, second key)
-    void* survivors;     // [kMaxSparseCtas][slices][256] survivor lists of the sparse walk
     // bucket walk: bit planes of the one-byte tokens by class, live classes of every state
-    uint32_t* planes;    // [256][W] bit v of plane c: token v is the one byte of class c
+    uint32_t* planes;    // [256][plane_stride(W)] bit v of plane c: token v is the one byte of class c
+    uint8_t* tok_c1;     // [N rounded up to 1024] class of a one-byte token, else the null class
     uint32_t* live;      // [Q][8] bit c: state reads class c
     int32_t* row_count;  // [Q] allowed tokens per row (compressed-row build)
     uint16_t* tok_head;  // [N] first byte | min(length, 255) << 8 of every token
@@ -54,10 +54,14 @@ struct Workspace {
     uint16_t* csr_dense; // [Q][N] end states of an automaton of fewer than kCsrDenseRows states
                          // (compressed-row build: the rows are cut out of the dense table)
     size_t bytes;        // everything above
-    size_t dense_bytes;  // the part in front of `survivors`: enough for the dense walk
+    size_t dense_bytes;  // the leading part that the dense walk needs
 };
 
 inline size_t table_elem_bytes(int32_t Q) { return Q <= 65535 ? 2 : 4; }
+
+// Words between the bit planes of two classes: the row length rounded up so that every
+// plane starts on a 16-byte boundary.
+__host__ __device__ constexpr int plane_stride(int W) { return (W + 3) & ~3; }
 
 // Row stride of the compressed table in entries: room for C classes and the null class,
 // and an odd number of 32-bit words, so that the same column of 32 different rows lies
@@ -83,23 +87,18 @@ inline Workspace carve(void* base, int32_t Q, int32_t N) {
     w.partial = reinterpret_cast<uint64_t*>(take(sizeof(uint64_t) * kHashBlocks * 256));
     w.table = take(static_cast<size_t>(Q) * kMaxCs * table_elem_bytes(Q));
     const size_t dense_bytes = G32 * sizeof(uint4) + G32;
-    const size_t srec_bytes = align_up(static_cast<size_t>(N) * sizeof(uint4), 256);
-    const size_t sparse_bytes = srec_bytes + static_cast<size_t>(N) * sizeof(int32_t);
-    uint8_t* tokens = take(dense_bytes > sparse_bytes ? dense_bytes : sparse_bytes);
+    uint8_t* tokens = take(dense_bytes);  // (the sorted records, N * 16 bytes, fit as well)
     w.tok_cls = reinterpret_cast<uint4*>(tokens);
     w.tok_len = tokens ? tokens + G32 * sizeof(uint4) : nullptr;
     w.srec = reinterpret_cast<uint4*>(tokens);
-    w.sid = reinterpret_cast<int32_t*>(tokens ? tokens + srec_bytes : nullptr);
     w.gstart = reinterpret_cast<int32_t*>(take(257 * sizeof(int32_t)));
     w.row_ctr = reinterpret_cast<int32_t*>(take(sizeof(int32_t)));
     w.count2 = reinterpret_cast<int32_t*>(take(kKeys * sizeof(int32_t)));
     w.cursor2 = reinterpret_cast<int32_t*>(take(kKeys * sizeof(int32_t)));
     w.start2 = reinterpret_cast<int32_t*>(take(kKeys * sizeof(int32_t)));
     w.dense_bytes = off;
-    const size_t ctas = Q < kMaxSparseCtas ? Q : kMaxSparseCtas;
-    const size_t slice_slots = (static_cast<size_t>(N) + 511) / 512 * 512;
-    w.survivors = take(ctas * slice_slots * (Q <= 65535 ? 4 : 8));
-    w.planes = reinterpret_cast<uint32_t*>(take(256 * (G32 / 32) * sizeof(uint32_t)));
+    w.planes = reinterpret_cast<uint32_t*>(take(256 * static_cast<size_t>(plane_stride(static_cast<int>(G32 / 32))) * sizeof(uint32_t)));
+    w.tok_c1 = take((static_cast<size_t>(N) + 1023) / 1024 * 1024);
     w.live = reinterpret_cast<uint32_t*>(take(static_cast<size_t>(Q) * 8 * sizeof(uint32_t)));
     w.row_count = reinterpret_cast<int32_t*>(take(static_cast<size_t>(Q) * sizeof(int32_t)));
     w.tok_head = reinterpret_cast<uint16_t*>(take(static_cast<size_t>(N) * sizeof(uint16_t)));
@@ -124,15 +123,15 @@ struct WalkParams {
     // dense walk
     const uint4* tok_cls;
     const uint8_t* tok_len;
-    // sparse walk
+    // work-avoiding walks
     const uint4* srec;
-    const int32_t* sid;
     const int32_t* gstart;
     const int32_t* count2;
     const int32_t* start2;
     int32_t* row_ctr;
     // bucket walk
     const uint32_t* planes;
+    const uint8_t* tok_c1;
     const uint32_t* live;
     const int32_t* row_order;  // row-wise walk: rows in the order they are handed out, or null
     const int32_t* win_order;  // bucket walk: windows in the order they are handed out, or null
@@ -155,7 +154,7 @@ __device__ __forceinline__ uint32_t clamp_state(int32_t v, int32_t Q, int32_t de
     return (static_cast<uint32_t>(v) >= static_cast<uint32_t>(Q)) ? dead : v;
 }
 
-// Bucket key of a token in the sorted order of the sparse walk.
+// Bucket key of a token in the sorted order of the work-avoiding walks.
 __device__ __forceinline__ int bucket_key(bool two_level, int first, int second_key) {
     return two_level ? first * kKeyStride + second_key : first;
 }
@@ -221,19 +220,19 @@ __device__ __forceinline__ uint32_t raw_walk(const WalkParams& p, uint32_t s, in
     return raw_walk_impl(p.trans, p.vocab_bytes, p.Q, p.dead, s, o0, o1, from);
 }
 
-// Bytes START.. of one token walked from state s, all 32 lanes in lock step.  `go`
+// Bytes START .. END-1 of one token walked from state s, all 32 lanes in lock step.  `go`
 // says whether this lane still has a live walk with bytes left.  The loop is
 // warp-uniform (one vote per byte) and its body has no branches: lanes that are done
 // keep their state through a select.  Every state value is a valid table row
 // (out-of-range entries were replaced by `dead` when the table was compressed), so the
 // shared-memory lookup needs no guard; the global-memory lookup is predicated to save
-// traffic.  On return `go` is true only for tokens longer than the inline record.
-template <typename TabT, bool FULL, int START>
+// traffic.  On return `go` is true only for tokens longer than the record covers.
+template <typename TabT, bool FULL, int START, int END = kInlineBytes>
 __device__ __forceinline__ uint32_t walk_rest(const TabT* __restrict__ tab, uint32_t Cs,
                                               uint32_t dead, const uint4& tk, int len, uint32_t s,
                                               bool& go) {
 #pragma unroll
-    for (int i = START; i < kInlineBytes; ++i) {
+    for (int i = START; i < END; ++i) {
         if (!__any_sync(kFullWarp, go)) break;
         const uint32_t c = tok_byte(tk, i);
         uint32_t ns;

@@ -141,7 +141,7 @@ prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab
             IndexMeta* meta, uint8_t* __restrict__ cls_out, TabT* __restrict__ table,
             uint4* __restrict__ tok_cls, uint8_t* __restrict__ tok_len,
             uint32_t* __restrict__ live, int32_t* __restrict__ count2, uint32_t* __restrict__ planes,
-            uint16_t* __restrict__ tok_head, int32_t* status) {
+            uint16_t* __restrict__ tok_head, uint8_t* __restrict__ tok_c1, int32_t* status) {
     extern __shared__ int s_cnt[];  // [kKeys] when keys are counted
     __shared__ ClassScratch cs;
     __shared__ uint8_t s_cls[256], s_rep[256];
@@ -241,7 +241,7 @@ prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab
     const int nchunks = (N + kPrepTokens - 1) / kPrepTokens;
     if (count2 != nullptr && static_cast<int>(blockIdx.x) < nchunks) {
         const int nkeys = two ? kKeys : 256;
-        const int W = (N + 31) / 32;
+        const int W = (N + 31) / 32, Wp = plane_stride(W);
         for (int i = tid; i < nkeys; i += kPrepThreads) s_cnt[i] = 0;
         bool bad = bad_tok;
         for (int chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
@@ -250,7 +250,7 @@ prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab
             if (planes != nullptr)
                 for (int i = tid; i < C * 32; i += kPrepThreads) {
                     const int word = chunk * 32 + (i & 31);
-                    if (word < W) planes[static_cast<size_t>(i >> 5) * W + word] = 0;
+                    if (word < Wp) planes[static_cast<size_t>(i >> 5) * Wp + word] = 0;
                 }
             __syncthreads();
             const int64_t v = static_cast<int64_t>(chunk) * kPrepTokens + tid;
@@ -260,12 +260,14 @@ prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab
             const TokenInfo t = token_classify(raw, s_cls);
             if (tok_head != nullptr && v < N)  // first byte and length, for the compressed rows
                 tok_head[v] = static_cast<uint16_t>(raw.b0 | (static_cast<uint32_t>(raw.len) << 8));
+            if (tok_c1 != nullptr)  // (the array is padded to whole passes)
+                tok_c1[v] = static_cast<uint8_t>(t.len == 1 ? t.first : C);
             if (t.len > 0) atomicAdd(&s_cnt[bucket_key(two, t.first, t.second_key)], 1);
             if (planes != nullptr) {
                 const bool one = t.len == 1;
                 const uint32_t peers = __match_any_sync(kFullWarp, one ? t.first : 0xFFFF);
                 if (one && (tid & 31) == __ffs(peers) - 1)
-                    planes[static_cast<size_t>(t.first) * W + (v >> 5)] = peers;
+                    planes[static_cast<size_t>(t.first) * Wp + (v >> 5)] = peers;
             }
         }
         if (__syncthreads_or(bad) && tid == 0) raise_flag(status, FSM_FLAG_OFFSETS);
@@ -281,7 +283,8 @@ prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab
 // publishes it, and the first position of every first class, for the walk).  Then the
 // blocks share the tokens, kPrepTokens at a time: rank within the pass by shared-memory
 // counters, one global atomic per key present in the pass to reserve its positions.  A
-// record keeps the length and the classes of bytes 1..15; `sid` holds the token id.
+// record keeps the length (capped at kSortedInline + 1), the classes of bytes
+// 1 .. kSortedInline - 1 and, in its last word, the token id.
 constexpr int kScanPer = (kKeys + kPrepThreads - 1) / kPrepThreads;  // keys per thread
 constexpr int kKeysPad = kScanPer * kPrepThreads;
 constexpr int kOrderBuckets = 2048;  // candidate-count buckets of the row order
@@ -290,7 +293,7 @@ __global__ void __launch_bounds__(kPrepThreads)
 sort_all(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vocab_offsets,
          int64_t vocab_nbytes, int32_t N, int32_t eos_id, const IndexMeta* meta,
          const uint8_t* cls, const int32_t* count2, int32_t* cursor2, int32_t* __restrict__ start2,
-         int32_t* __restrict__ gstart, uint4* __restrict__ srec, int32_t* __restrict__ sid,
+         int32_t* __restrict__ gstart, uint4* __restrict__ srec,
          const uint32_t* live, int32_t q_begin, int32_t q_end, int32_t* row_order,
          int32_t* win_order) {
     extern __shared__ int s_sort[];  // s_start[kKeysPad], s_cnt[kKeys]
@@ -303,9 +306,9 @@ sort_all(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vo
     bool bad_first = false;
     const TokenRaw raw_first = token_raw(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id,
                                          static_cast<int64_t>(blockIdx.x) * kPrepTokens + tid, &bad_first);
-    uint8_t bytes_first[kInlineBytes];
+    uint8_t bytes_first[kSortedInline];
 #pragma unroll
-    for (int i = 2; i < kInlineBytes; ++i)
+    for (int i = 2; i < kSortedInline; ++i)
         bytes_first[i] = i < raw_first.len ? vocab_bytes[raw_first.start + i] : 0;
     bytes_first[0] = static_cast<uint8_t>(raw_first.b0);
     bytes_first[1] = static_cast<uint8_t>(raw_first.b1);
@@ -466,9 +469,9 @@ sort_all(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vo
         const int key = t.len > 0 ? bucket_key(two, t.first, t.second_key) : 0;
         int rank = 0;
         if (t.len > 0) rank = atomicAdd(&s_cnt[key], 1);
-        uint8_t bytes[kInlineBytes];
+        uint8_t bytes[kSortedInline];
 #pragma unroll
-        for (int i = 1; i < kInlineBytes; ++i) {  // independent loads, issued together
+        for (int i = 1; i < kSortedInline; ++i) {  // independent loads, issued together
             if (first)
                 bytes[i] = bytes_first[i];
             else
@@ -498,13 +501,12 @@ sort_all(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vo
         __syncthreads();
         if (t.len > 0) {
             const int pos = s_cnt[key] + rank;
-            uint32_t w[4] = {static_cast<uint32_t>(t.len), 0, 0, 0};
-            const int nb = min(t.len, kInlineBytes);
+            uint32_t w[3] = {static_cast<uint32_t>(min(t.len, kSortedInline + 1)), 0, 0};
+            const int nb = min(t.len, kSortedInline);
 #pragma unroll
-            for (int i = 1; i < kInlineBytes; ++i)
+            for (int i = 1; i < kSortedInline; ++i)
                 if (i < nb) w[i >> 2] |= static_cast<uint32_t>(s_cls[bytes[i]]) << ((i & 3) * 8);
-            srec[pos] = make_uint4(w[0], w[1], w[2], w[3]);
-            sid[pos] = static_cast<int32_t>(v);
+            srec[pos] = make_uint4(w[0], w[1], w[2], static_cast<uint32_t>(v));
         }
     }
 }
