@@ -96,11 +96,11 @@ size_t fsm_index_workspace_bytes(int32_t Q, int32_t N, int64_t vocab_nbytes);
  *   state_dtype    FSM_STATE_I32, or FSM_STATE_U16 (requires Q <= 65535).
  *   workspace      device scratch, 256-byte aligned, at least
  *                  fsm_index_workspace_bytes(Q, N, vocab_nbytes) bytes (the compressed
- *                  table, the token records and, for the work-avoiding walk, per-CTA
- *                  survivor lists of min(Q,160) * N entries: about 85 MB for 1,001
- *                  states and 128,256 tokens; for Q < 256 also Q * N 16-bit entries,
- *                  from which fsm_index_build_csr cuts its rows).  Contents on entry
- *                  are irrelevant; concurrent calls need separate workspaces.
+ *                  table, the token records, the bit planes of the one-byte tokens:
+ *                  about 7 MB for 1,001 states and 128,256 tokens; for Q < 256 also
+ *                  Q * N 16-bit entries, from which fsm_index_build_csr cuts its rows).
+ *                  Contents on entry are irrelevant; concurrent calls need separate
+ *                  workspaces.
  *   status_word    device int32 or NULL.
  *
  * fsm_index_build_rows builds only rows q_begin <= q < q_end, written to
@@ -282,16 +282,16 @@ int guided_step_csr(const void* logits_in, void* logits_out, int32_t logits_dtyp
                                        byte-class verification fails and the exact
                                        uncompressed path is exercised */
 #define FSM_TUNE_MASK_CLUSTER 2     /* CTAs per logits row in guided_mask_step: 1,2,4,8; 0 = auto */
-#define FSM_TUNE_WALK_CTAS 3        /* CTAs of the walk kernel; 0 = one per SM */
+#define FSM_TUNE_WALK_CTAS 3        /* CTAs of the preparation and walk kernels; 0 = one per SM */
 #define FSM_TUNE_SMEM_TABLE_BYTES 4 /* cap on the shared-memory table tile; 0 = device maximum */
 #define FSM_PROFILE_WALK 5          /* non-zero: record a CUDA event pair around the walk
                                        kernel of every index build (see fsm_profile_read) */
 #define FSM_TUNE_WALK_ALGO 6        /* 0 = automatic (a build of at least one row per SM: 2
                                        with a next-state table, 3 without; a smaller one: 1),
-                                       1 = dense warp-tile walk, 2 = row-wise work-avoiding
+                                       1 = dense warp-tile walk, 2 = row-wise fill-and-patch
                                        walk, 3 = bucket walk (bitmask-only builds; builds with
-                                       a next-state table fall back to 1).  Same results in
-                                       every case */
+                                       a next-state table take 2).  Same results in every
+                                       case */
 int fsm_debug_set(int32_t key, int32_t value);
 
 /*

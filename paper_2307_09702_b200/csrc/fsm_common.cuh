@@ -54,24 +54,19 @@ cudaError_t launch_on(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sm
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-// Launch with programmatic stream serialisation: the kernel's blocks may become resident
-// while the preceding kernel of the stream is still running (once all of that kernel's
-// blocks have called pdl_launch_dependents()).  Such a kernel reads nothing an earlier
-// kernel writes, and writes nothing, before it has called pdl_wait(); and it reads what an
-// earlier kernel wrote through plain pointers only - a load through a `const __restrict__`
-// pointer or __ldg() counts as invariant for the whole kernel and may be moved in front of
-// the wait.  Used for the preparation kernels, whose first loads are inputs of the build.
+// Cooperative launch: every block of the grid is resident at once (the launch fails
+// otherwise), so the kernel may use grid-wide barriers.
 template <typename... KArgs, typename... Args>
-cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
-                              cudaStream_t stream, Args&&... args) {
+cudaError_t launch_cooperative(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                               cudaStream_t stream, Args&&... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
@@ -79,14 +74,6 @@ cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 #endif
 
 #ifdef __CUDACC__
-// Waits until the kernels launched before this one in the stream have completed and their
-// writes are visible (returns at once in a kernel that was launched the plain way).
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-// Lets the next kernel of the stream become resident once every block has got here.
-__device__ __forceinline__ void pdl_launch_dependents() {
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-}
-
 __device__ __forceinline__ void raise_flag(int32_t* status_word, int flag) {
     if (status_word != nullptr) atomicOr(status_word, flag);
 }

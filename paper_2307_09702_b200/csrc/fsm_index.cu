@@ -2,17 +2,18 @@
 // host entry points.  The kernels live in the fsm_index_*.cuh headers.
 //
 // Launches on the caller's stream, no host synchronisation:
-//   1. hash_columns    one pass over delta: a 64-bit hash of each of the 256 byte columns
-//   2. prepare_all     bytes with equal column hashes share a byte class; class-compressed
-//                      table [Q x Cs] with exact verification that every byte's column
-//                      equals its class representative's column; token records (dense
-//                      walk) or bucket key counts (work-avoiding walks)
-//   3. sort_all        work-avoiding walks only: tokens sorted by (first, second) byte class
-//   4. walk            dense: every (state, token) pair walked by warp tiles;
+//   1. prepare_fused   (cooperative, three phases with grid barriers in between)
+//        hash     one pass over delta: a 64-bit hash of each of the 256 byte columns
+//        prepare  bytes with equal column hashes share a byte class; class-compressed
+//                 table [Q x Cs] with exact verification that every byte's column
+//                 equals its class representative's column; token records (dense
+//                 walk) or bucket key counts (work-avoiding walks)
+//        sort     work-avoiding walks only: tokens sorted by (first, second) byte class
+//   2. walk            dense: every (state, token) pair walked by warp tiles;
 //      walk_rows       rows filled from a per-row table, longer tokens of readable buckets
 //                      walked and patched in;
 //      mask_onebyte + walk_buckets   bitmask-only builds
-// If verification in 2 fails (a 64-bit hash collision) the walk reads the uncompressed
+// If the verification fails (a 64-bit hash collision) the walk reads the uncompressed
 // table instead, so the result is exact in every case.
 #include "fsm_index_common.cuh"
 #include "fsm_index_dense.cuh"
@@ -75,62 +76,64 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     const bool bucket = next_state == nullptr && !dense_only &&
                         (tune.walk_algo == 3 || (tune.walk_algo == 0 && enough_rows));
     const bool rows = !bucket && rows_fits &&
-                      (tune.walk_algo == 2 || (tune.walk_algo == 0 && enough_rows));
+                      (tune.walk_algo == 2 || tune.walk_algo == 3 || (tune.walk_algo == 0 && enough_rows));
     const bool sparse = bucket || rows;  // tokens sorted by bucket key
 
-    const int hash_blocks = Q < kHashBlocks ? Q : kHashBlocks;
-    if (launch_overlapped(hash_columns, dim3(hash_blocks), dim3(256 * kHashRowLanes), 0, stream,
-                          dfa_trans, Q, dead_state, ws.partial, tune.weak_hash, ws.meta,
-                          ws.count2, ws.cursor2, ws.row_ctr, status_word) != cudaSuccess)
-        return FSM_ERR_CUDA;
-    // prepare_all: blocks share the table rows and the tokens
-    const int nchunks = (N + kPrepTokens - 1) / kPrepTokens;
-    const int row_passes = (Q + kPrepRows - 1) / kPrepRows;
-    int prep_blocks = row_passes > nchunks ? row_passes : nchunks;
-    if (prep_blocks > dev.sm_count) prep_blocks = dev.sm_count;
-    uint4* tok_cls = sparse ? nullptr : ws.tok_cls;  // dense walk: token records
-    int32_t* count2 = sparse ? ws.count2 : nullptr;  // work-avoiding walks: bucket keys
-    uint32_t* live = sparse ? ws.live : nullptr;  // bucket walk; row order of the row-wise walk
+    // ---- preparation: one cooperative launch, one block per SM
     int32_t* row_order = sparse && !bucket ? ws.row_order : nullptr;
     // (the ranking of the windows counts them in kKeys words of shared memory)
-    int32_t* win_order = bucket && sparse && (N + 31) / 32 <= kKeys ? ws.win_order : nullptr;
-    uint32_t* planes = bucket || rows ? ws.planes : nullptr;
-    uint8_t* tok_c1 = rows ? ws.tok_c1 : nullptr;
-    const size_t key_smem = sparse ? kKeys * sizeof(int) : 0;
-    const size_t sort_smem = (kKeysPad + kKeys) * sizeof(int);
-    if (wide) {
-        auto k = prepare_all<int32_t>;
-        if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(kKeys * sizeof(int))) != cudaSuccess)
-            return FSM_ERR_CUDA;
-        if (launch_overlapped(k, dim3(prep_blocks), dim3(kPrepThreads), key_smem, stream, dfa_trans,
-                              vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
-                              ws.partial, hash_blocks, ws.meta, ws.cls, static_cast<int32_t*>(ws.table),
-                              tok_cls, ws.tok_len, live, count2, planes,
-                              want_tok_head ? ws.tok_head : nullptr, tok_c1, status_word) != cudaSuccess)
-            return FSM_ERR_CUDA;
-    } else {
-        auto k = prepare_all<uint16_t>;
-        if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(kKeys * sizeof(int))) != cudaSuccess)
-            return FSM_ERR_CUDA;
-        if (launch_overlapped(k, dim3(prep_blocks), dim3(kPrepThreads), key_smem, stream, dfa_trans,
-                              vocab_bytes, vocab_offsets, vocab_nbytes, Q, N, dead_state, eos_id,
-                              ws.partial, hash_blocks, ws.meta, ws.cls, static_cast<uint16_t*>(ws.table),
-                              tok_cls, ws.tok_len, live, count2, planes,
-                              want_tok_head ? ws.tok_head : nullptr, tok_c1, status_word) != cudaSuccess)
-            return FSM_ERR_CUDA;
-    }
-    if (sparse) {
-        if (cudaFuncSetAttribute(sort_all, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(sort_smem)) != cudaSuccess)
-            return FSM_ERR_CUDA;
-        const int sort_blocks = nchunks < dev.sm_count ? nchunks : dev.sm_count;
-        if (launch_overlapped(sort_all, dim3(sort_blocks + (row_order || win_order ? 1 : 0)), dim3(kPrepThreads),
-                              sort_smem, stream, vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id,
-                              ws.meta, ws.cls, ws.count2, ws.cursor2, ws.start2, ws.gstart, ws.srec,
-                              live, q_begin, q_end, row_order, win_order) != cudaSuccess)
-            return FSM_ERR_CUDA;
+    int32_t* win_order = bucket && (N + 31) / 32 <= kKeys ? ws.win_order : nullptr;
+    {
+        PrepParams a = {};
+        a.trans = dfa_trans;
+        a.vocab_bytes = vocab_bytes;
+        a.vocab_offsets = vocab_offsets;
+        a.vocab_nbytes = vocab_nbytes;
+        a.Q = Q;
+        a.N = N;
+        a.dead = dead_state;
+        a.eos_id = eos_id;
+        a.q_begin = q_begin;
+        a.q_end = q_end;
+        a.nparts = Q < kHashBlocks ? Q : kHashBlocks;
+        a.weak = tune.weak_hash;
+        a.sorted = sparse ? 1 : 0;
+        a.partial = ws.partial;
+        a.meta = ws.meta;
+        a.cls = ws.cls;
+        a.table = ws.table;
+        a.tok_cls = ws.tok_cls;  // dense walk: token records
+        a.tok_len = ws.tok_len;
+        a.live = sparse ? ws.live : nullptr;  // bucket walk; row order of the row-wise walk
+        a.count2 = ws.count2;
+        a.cursor2 = ws.cursor2;
+        a.start2 = ws.start2;
+        a.gstart = ws.gstart;
+        a.row_ctr = ws.row_ctr;
+        a.planes = bucket || rows ? ws.planes : nullptr;
+        a.tok_head = want_tok_head ? ws.tok_head : nullptr;
+        a.tok_c1 = rows ? ws.tok_c1 : nullptr;
+        a.srec = ws.srec;
+        a.row_order = row_order;
+        a.win_order = win_order;
+        a.status = status_word;
+        const size_t prep_smem = (sparse ? kKeysPad + kKeys : 0) * sizeof(int);
+        int prep_blocks = dev.sm_count;
+        if (tune.walk_ctas > 0 && tune.walk_ctas < prep_blocks) prep_blocks = tune.walk_ctas;
+        if (prep_blocks < a.nparts) a.nparts = prep_blocks;
+        cudaError_t e;
+        if (wide) {
+            auto k = prepare_fused<int32_t>;
+            e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(prep_smem));
+            if (e == cudaSuccess)
+                e = launch_cooperative(k, dim3(prep_blocks), dim3(kPrepThreads), prep_smem, stream, a);
+        } else {
+            auto k = prepare_fused<uint16_t>;
+            e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(prep_smem));
+            if (e == cudaSuccess)
+                e = launch_cooperative(k, dim3(prep_blocks), dim3(kPrepThreads), prep_smem, stream, a);
+        }
+        if (e != cudaSuccess) return FSM_ERR_CUDA;
     }
     if (cudaGetLastError() != cudaSuccess) return FSM_ERR_CUDA;
 

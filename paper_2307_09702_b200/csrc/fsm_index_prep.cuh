@@ -1,11 +1,14 @@
-// Preparation kernels of the index build: byte classes, compressed table, token layouts.
+// Preparation of the index build: byte classes, compressed table, token layouts.
 //
-// Three launches: hash_columns (a hash of each byte column of delta), prepare_all (every
-// block derives the byte classes from the hashes, then the blocks share the table rows and
-// the tokens) and, for the work-avoiding walks, sort_all (every block scans the key counts,
+// One cooperative launch (one block per SM, all resident) in three phases separated by grid
+// barriers: hash_phase (a hash of each byte column of delta), prepare_phase (every block
+// derives the byte classes from the hashes, then the blocks share the table rows and the
+// tokens) and, for the work-avoiding walks, sort_phase (every block scans the key counts,
 // then the blocks share the tokens).  The small serial steps are repeated by every block
-// instead of being launches of their own.
+// instead of being phases of their own.
 #pragma once
+
+#include <cooperative_groups.h>
 
 #include "fsm_index_common.cuh"
 
@@ -19,25 +22,14 @@ namespace {
 // blocks also clear the counters of the token sort and the flag of the class check.
 constexpr int kHashRowLanes = 4;
 
-__global__ void __launch_bounds__(256 * kHashRowLanes)
-hash_columns(const int32_t* __restrict__ trans, int32_t Q, int32_t dead,
-             uint64_t* __restrict__ partial, int weak, IndexMeta* meta,
-             int32_t* __restrict__ count2,
-             int32_t* __restrict__ cursor2, int32_t* __restrict__ row_ctr, int32_t* status) {
+// (`nparts` blocks hash; every block helps clear the counters.)
+__device__ __forceinline__ void hash_phase(const int32_t* __restrict__ trans, int32_t Q, int32_t dead,
+                                           uint64_t* __restrict__ partial, int nparts, int weak,
+                                           IndexMeta* meta, int32_t* __restrict__ count2,
+                                           int32_t* __restrict__ cursor2, int32_t* __restrict__ row_ctr,
+                                           int32_t* status) {
     __shared__ uint64_t part[kHashRowLanes][256];
     const int b = threadIdx.x & 255, rl = threadIdx.x >> 8;
-    pdl_launch_dependents();
-    // delta is an input of the build: it may be read while the previous kernel still runs
-    uint64_t h = 0;
-    bool bad = false;
-#pragma unroll 4
-    for (int q = blockIdx.x * kHashRowLanes + rl; q < Q; q += gridDim.x * kHashRowLanes) {
-        const int32_t v = trans[static_cast<size_t>(q) * 256 + b];
-        if (q == dead) continue;
-        bad |= static_cast<uint32_t>(v) >= static_cast<uint32_t>(Q);
-        h += mix64((static_cast<uint64_t>(q) << 32) | static_cast<uint32_t>(v));
-    }
-    pdl_wait();  // the workspace may still be in use by the kernels before this one
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         *row_ctr = 0;
         meta->any_bad = 0;
@@ -45,6 +37,16 @@ hash_columns(const int32_t* __restrict__ trans, int32_t Q, int32_t dead,
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < kKeys; i += gridDim.x * blockDim.x) {
         count2[i] = 0;
         cursor2[i] = 0;
+    }
+    if (static_cast<int>(blockIdx.x) >= nparts) return;
+    uint64_t h = 0;
+    bool bad = false;
+#pragma unroll 4
+    for (int q = blockIdx.x * kHashRowLanes + rl; q < Q; q += nparts * kHashRowLanes) {
+        const int32_t v = trans[static_cast<size_t>(q) * 256 + b];
+        if (q == dead) continue;
+        bad |= static_cast<uint32_t>(v) >= static_cast<uint32_t>(Q);
+        h += mix64((static_cast<uint64_t>(q) << 32) | static_cast<uint32_t>(v));
     }
     part[rl][b] = h;
     const int any_bad = __syncthreads_or(bad);
@@ -134,31 +136,19 @@ __device__ __forceinline__ int derive_classes(const uint64_t* partial, int npart
 //     start with a space are a third of a BPE vocabulary and would otherwise all hit the
 //     same few counters.
 template <typename TabT>
-__global__ void __launch_bounds__(kPrepThreads)
-prepare_all(const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab_bytes,
-            const int32_t* __restrict__ vocab_offsets, int64_t vocab_nbytes, int32_t Q, int32_t N,
-            int32_t dead, int32_t eos_id, const uint64_t* partial, int nparts,
-            IndexMeta* meta, uint8_t* __restrict__ cls_out, TabT* __restrict__ table,
-            uint4* __restrict__ tok_cls, uint8_t* __restrict__ tok_len,
-            uint32_t* __restrict__ live, int32_t* __restrict__ count2, uint32_t* __restrict__ planes,
-            uint16_t* __restrict__ tok_head, uint8_t* __restrict__ tok_c1, int32_t* status) {
-    extern __shared__ int s_cnt[];  // [kKeys] when keys are counted
+__device__ __forceinline__ void prepare_phase(
+    const int32_t* __restrict__ trans, const uint8_t* __restrict__ vocab_bytes,
+    const int32_t* __restrict__ vocab_offsets, int64_t vocab_nbytes, int32_t Q, int32_t N, int32_t dead,
+    int32_t eos_id, const uint64_t* partial, int nparts, IndexMeta* meta, uint8_t* __restrict__ cls_out,
+    TabT* __restrict__ table, uint4* __restrict__ tok_cls, uint8_t* __restrict__ tok_len,
+    uint32_t* __restrict__ live, int32_t* __restrict__ count2, uint32_t* __restrict__ planes,
+    uint16_t* __restrict__ tok_head, uint8_t* __restrict__ tok_c1, int32_t* status,
+    int* s_cnt /* [kKeys] when keys are counted */, int32_t row_first, const TokenRaw& raw_first,
+    bool bad_tok) {
     __shared__ ClassScratch cs;
     __shared__ uint8_t s_cls[256], s_rep[256];
     __shared__ int32_t rows[kPrepRows][256];
     const int tid = threadIdx.x;
-    // What does not depend on the classes is fetched first: the block's first pass of table
-    // rows and of tokens.
-    int32_t row_first = dead;
-    if (static_cast<int>(blockIdx.x) * kPrepRows + (tid >> 8) < Q)
-        row_first = trans[(static_cast<size_t>(blockIdx.x) * kPrepRows + (tid >> 8)) * 256 + (tid & 255)];
-    bool bad_tok = false;
-    TokenRaw raw_first = {0, 0, 0, 0};
-    if (count2 != nullptr)
-        raw_first = token_raw(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id,
-                              static_cast<int64_t>(blockIdx.x) * kPrepTokens + tid, &bad_tok);
-    pdl_launch_dependents();
-    pdl_wait();  // the column hashes come from the kernel before
     const int C = derive_classes(partial, nparts, cs, s_cls, s_rep);
     const int Cs = table_row_stride<TabT>(C);
     const bool two = C <= kTwoLevelMaxC;
@@ -289,31 +279,18 @@ constexpr int kScanPer = (kKeys + kPrepThreads - 1) / kPrepThreads;  // keys per
 constexpr int kKeysPad = kScanPer * kPrepThreads;
 constexpr int kOrderBuckets = 2048;  // candidate-count buckets of the row order
 
-__global__ void __launch_bounds__(kPrepThreads)
-sort_all(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vocab_offsets,
-         int64_t vocab_nbytes, int32_t N, int32_t eos_id, const IndexMeta* meta,
-         const uint8_t* cls, const int32_t* count2, int32_t* cursor2, int32_t* __restrict__ start2,
-         int32_t* __restrict__ gstart, uint4* __restrict__ srec,
-         const uint32_t* live, int32_t q_begin, int32_t q_end, int32_t* row_order,
-         int32_t* win_order) {
-    extern __shared__ int s_sort[];  // s_start[kKeysPad], s_cnt[kKeys]
+__device__ __forceinline__ void sort_phase(
+    const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vocab_offsets,
+    int64_t vocab_nbytes, int32_t N, int32_t eos_id, const IndexMeta* meta, const uint8_t* cls,
+    const int32_t* count2, int32_t* cursor2, int32_t* __restrict__ start2, int32_t* __restrict__ gstart,
+    uint4* __restrict__ srec, const uint32_t* live, int32_t q_begin, int32_t q_end, int32_t* row_order,
+    int32_t* win_order, int* s_sort /* s_start[kKeysPad], s_cnt[kKeys] */, const TokenRaw& raw_first,
+    const uint8_t (&bytes_first)[kSortedInline]) {
     int* s_start = s_sort;
     int* s_cnt = s_sort + kKeysPad;
     __shared__ int wsum[kPrepThreads / 32];
     __shared__ uint8_t s_cls[256];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // the block's first pass of tokens does not depend on the scan: fetch its bytes first
-    bool bad_first = false;
-    const TokenRaw raw_first = token_raw(vocab_bytes, vocab_offsets, vocab_nbytes, N, eos_id,
-                                         static_cast<int64_t>(blockIdx.x) * kPrepTokens + tid, &bad_first);
-    uint8_t bytes_first[kSortedInline];
-#pragma unroll
-    for (int i = 2; i < kSortedInline; ++i)
-        bytes_first[i] = i < raw_first.len ? vocab_bytes[raw_first.start + i] : 0;
-    bytes_first[0] = static_cast<uint8_t>(raw_first.b0);
-    bytes_first[1] = static_cast<uint8_t>(raw_first.b1);
-    pdl_launch_dependents();
-    pdl_wait();  // classes and key counts come from the kernel before
     if (tid < 256) s_cls[tid] = cls[tid];
     const bool two = meta->two_level != 0;
     const int nkeys = two ? kKeys : 256;
@@ -509,6 +486,78 @@ sort_all(const uint8_t* __restrict__ vocab_bytes, const int32_t* __restrict__ vo
             srec[pos] = make_uint4(w[0], w[1], w[2], static_cast<uint32_t>(v));
         }
     }
+}
+
+// ---------------------------------------------------------------------------- fused
+// The whole preparation as one cooperative kernel (one block per SM).  The blocks fetch
+// what depends on the build's inputs only (their first table rows, their first tokens)
+// before the first grid barrier.
+struct PrepParams {
+    const int32_t* trans;
+    const uint8_t* vocab_bytes;
+    const int32_t* vocab_offsets;
+    int64_t vocab_nbytes;
+    int32_t Q, N, dead, eos_id, q_begin, q_end;
+    int nparts;  // blocks that hash table rows
+    int weak;
+    int sorted;  // tokens are sorted by bucket key (work-avoiding walks)
+    uint64_t* partial;
+    IndexMeta* meta;
+    uint8_t* cls;
+    void* table;
+    uint4* tok_cls;
+    uint8_t* tok_len;
+    uint32_t* live;
+    int32_t* count2;
+    int32_t* cursor2;
+    int32_t* start2;
+    int32_t* gstart;
+    int32_t* row_ctr;
+    uint32_t* planes;
+    uint16_t* tok_head;
+    uint8_t* tok_c1;
+    uint4* srec;
+    int32_t* row_order;
+    int32_t* win_order;
+    int32_t* status;
+};
+
+template <typename TabT>
+__global__ void __launch_bounds__(kPrepThreads, 1) prepare_fused(const PrepParams a) {
+    extern __shared__ int s_dyn[];  // key counters (prepare), scan + counters (sort)
+    namespace cg = cooperative_groups;
+    cg::grid_group grid = cg::this_grid();
+    const int tid = threadIdx.x;
+    // ---- inputs of the build, fetched before anything else is known
+    int32_t row_first = a.dead;
+    if (static_cast<int>(blockIdx.x) * kPrepRows + (tid >> 8) < a.Q)
+        row_first = a.trans[(static_cast<size_t>(blockIdx.x) * kPrepRows + (tid >> 8)) * 256 + (tid & 255)];
+    bool bad_tok = false;
+    TokenRaw raw_first = {0, 0, 0, 0};
+    uint8_t bytes_first[kSortedInline];
+#pragma unroll
+    for (int i = 0; i < kSortedInline; ++i) bytes_first[i] = 0;
+    if (a.sorted) {
+        raw_first = token_raw(a.vocab_bytes, a.vocab_offsets, a.vocab_nbytes, a.N, a.eos_id,
+                              static_cast<int64_t>(blockIdx.x) * kPrepTokens + tid, &bad_tok);
+#pragma unroll
+        for (int i = 2; i < kSortedInline; ++i)
+            bytes_first[i] = i < raw_first.len ? a.vocab_bytes[raw_first.start + i] : 0;
+        bytes_first[0] = static_cast<uint8_t>(raw_first.b0);
+        bytes_first[1] = static_cast<uint8_t>(raw_first.b1);
+    }
+    hash_phase(a.trans, a.Q, a.dead, a.partial, a.nparts, a.weak, a.meta, a.count2, a.cursor2, a.row_ctr,
+               a.status);
+    grid.sync();
+    prepare_phase<TabT>(a.trans, a.vocab_bytes, a.vocab_offsets, a.vocab_nbytes, a.Q, a.N, a.dead, a.eos_id,
+                        a.partial, a.nparts, a.meta, a.cls, static_cast<TabT*>(a.table),
+                        a.sorted ? nullptr : a.tok_cls, a.tok_len, a.live, a.sorted ? a.count2 : nullptr,
+                        a.planes, a.tok_head, a.tok_c1, a.status, s_dyn, row_first, raw_first, bad_tok);
+    if (!a.sorted) return;
+    grid.sync();
+    sort_phase(a.vocab_bytes, a.vocab_offsets, a.vocab_nbytes, a.N, a.eos_id, a.meta, a.cls, a.count2,
+               a.cursor2, a.start2, a.gstart, a.srec, a.live, a.q_begin, a.q_end, a.row_order, a.win_order,
+               s_dyn, raw_first, bytes_first);
 }
 
 }  // namespace
