@@ -36,13 +36,12 @@ if ROOT not in sys.path:
 METRIC = "index build (state,token) walks/s; masked-logit step us at B=256, N=128k"
 UNIT = "walks/s"
 B_ROWS = 256
-SMEM_LOOKUP_BOUND = 148 * 32 * 1.965e9 / 1.157
-# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/
-# (walk_sparse_config3.md, mask_step_config5.md).  Set an entry to None when the kernel
-# changes and the capture has not been redone.
-NCU_TRAFFIC = {"walk_sparse": 506_000_000, "mask_step": 68_600_000}
-# kernels of this library per timed step: hash_columns, prepare_all, sort_all, walk_sparse,
-# mask_step
+# DRAM bytes (read + write) per launch come from the ncu summaries under profiles/: each
+# names the kernel source it was captured from with that file's SHA-256, and a summary whose
+# source has changed since gives no figure (see ncu_traffic()).
+PROFILES = {"walk_rows": "walk_rows_config3.md", "mask_step": "mask_step_config5.md"}
+# kernels of this library per timed step: prepare_fused, walk_rows, mask_step
+LAUNCHES_PER_STEP = 3
 RING = 8
 
 
@@ -54,6 +53,52 @@ def load_peaks():
         return float(p["hbm_gbs"]), "measured"
     except Exception:
         return 6650.0, "fallback"
+
+
+def ncu_traffic(kind: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum of the first captured launch in the
+    profile summary of `kind`, or None when there is no summary or the kernel's source file
+    is no longer the one the capture was taken from."""
+    import hashlib
+    import re
+    path = os.path.join(ROOT, "profiles", PROFILES[kind])
+    try:
+        text = open(path).read()
+    except OSError:
+        return None
+    m = re.search(r"source:\s*(\S+)\s+sha256=([0-9a-f]+)", text)
+    if not m:
+        return None
+    try:
+        digest = hashlib.sha256(open(os.path.join(ROOT, m.group(1)), "rb").read()).hexdigest()
+    except OSError:
+        return None
+    if not digest.startswith(m.group(2)):
+        return None
+    scale = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
+    total = 0.0
+    for name in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
+        row = re.search(r"^\|\s*" + re.escape(name) + r"\s*\|\s*(\w+)\s*\|\s*([0-9.eE+-]+)", text, re.M)
+        if not row or row.group(1) not in scale:
+            return None
+        total += float(row.group(2)) * scale[row.group(1)]
+    return total
+
+
+def lookups_per_walk(w, threads, n_states=48):
+    """Table look-ups an early-exit walk makes per (state, token) pair, counted by the oracle
+    on a sample of the states (spread over the automaton)."""
+    from oracle import fsm_oracle
+    d = w.dfa
+    total, pairs = 0, 0
+    step = max(1, d.Q // n_states)
+    for q in range(0, d.Q, step):
+        _, _, n = fsm_oracle.index_build(d.trans, d.accept, w.vocab_bytes, w.vocab_offsets, d.dead,
+                                         w.eos_id, q_begin=q, q_end=q + 1, want_next=False,
+                                         threads=threads)
+        total += int(n)
+        pairs += w.N
+    return total / pairs
 
 
 def workload(rank: int):
@@ -332,8 +377,10 @@ def run_ours(args):
     walk_ms_mean = float(np.mean(walk_ms)) if walk_ms else float("nan")
 
     # ---- the other output modes of the index build (not part of the timed step)
-    def time_build(state_dtype, want_next, n=20):
-        other = fg.GuidedIndex(d.trans, d.accept, w.vocab_bytes, w.vocab_offsets, d.dead, w.eos_id,
+    def time_build(state_dtype, want_next, n=20, wl=None):
+        wl = wl or w
+        dd = wl.dfa
+        other = fg.GuidedIndex(dd.trans, dd.accept, wl.vocab_bytes, wl.vocab_offsets, dd.dead, wl.eos_id,
                                state_dtype, want_next, device=dev)
         for _ in range(3):
             other.build()
@@ -344,6 +391,7 @@ def run_ours(args):
             other.build()
         b.record()
         torch.cuda.synchronize()
+        assert int(other.status.item()) == 0
         return a.elapsed_time(b) / n
 
     u16_ms = time_build(fg.FSM_STATE_U16, True)
@@ -433,6 +481,83 @@ def run_ours(args):
 
     walks = float(w.Q) * w.N
     hbm_gbs, peak_kind = load_peaks()
+    # ---- bounds derived from this run: SM count, the SM clock sampled under load, and the
+    # look-ups per walk the oracle counts on a sample of the states
+    threads = len(os.sched_getaffinity(0))
+    sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+    sm_hz = 1e6 * float(clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0)
+
+    def lookup_bound(wl):
+        lpw = lookups_per_walk(wl, threads)
+        return sm_count * 32 * sm_hz / lpw, lpw
+
+    def build_modes(wl, t_i32, t_u16, t_mask, rated, why=None):
+        n_walks = float(wl.Q) * wl.N
+        bound, lpw = lookup_bound(wl)
+        out = {
+            "Q": wl.Q, "N": wl.N, "walks": n_walks, "sha256": wl.sha256(),
+            "lookups_per_walk": lpw,
+            "smem_lookup_bound_walks_per_s": bound,
+            "bound_inputs": {"sms": sm_count, "lookups_per_clk_per_sm": 32, "sm_mhz": sm_hz / 1e6},
+            "int32_states": {"us": t_i32 * 1e3, "walks_per_s": n_walks / (t_i32 * 1e-3),
+                             "hbm_write_bound_frac": (n_walks * 4.125 / (t_i32 * 1e-3) / 1e9) / hbm_gbs},
+            "uint16_states": {"us": t_u16 * 1e3, "walks_per_s": n_walks / (t_u16 * 1e-3),
+                              "hbm_write_bound_frac": (n_walks * 2.125 / (t_u16 * 1e-3) / 1e9) / hbm_gbs},
+            "bitmask_only": {"us": t_mask * 1e3, "walks_per_s": n_walks / (t_mask * 1e-3),
+                             "smem_lookup_bound_frac": (n_walks / (t_mask * 1e-3)) / bound},
+            "rated": rated,
+        }
+        if why:
+            out["note"] = why
+        return out
+
+    configs = {}
+    if world == 1 and not args.no_configs:
+        from fsm_inputs import make_config, step_logits_numpy
+        # workload 1: the whole build and 20 greedy steps at B = 1, fp32
+        w1 = make_config(1)
+        t1 = [time_build(sd, nx, wl=w1) for sd, nx in ((fg.FSM_STATE_I32, True), (fg.FSM_STATE_U16, True),
+                                                       (fg.FSM_STATE_I32, False))]
+        configs["1_tiny"] = build_modes(w1, *t1, rated=False,
+                                        why="6 states x 1,000 tokens: launch latency, not rated")
+        i1 = fg.GuidedIndex(w1.dfa.trans, w1.dfa.accept, w1.vocab_bytes, w1.vocab_offsets, w1.dfa.dead,
+                            w1.eos_id, device=dev).build()
+        x1 = [torch.from_numpy(step_logits_numpy(w1, i)).to(dev) for i in range(w1.steps)]
+        s1 = torch.zeros(1, dtype=torch.int32, device=dev)
+        f1 = torch.zeros(1, dtype=torch.uint8, device=dev)
+        k1 = torch.zeros(1, dtype=torch.int32, device=dev)
+        for rep in range(3):
+            s1.zero_()
+            f1.zero_()
+            xs = [x.clone() for x in x1]  # masked in place
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record()
+            for i in range(w1.steps):
+                i1.step(xs[i], s1, f1, k1)
+            b.record()
+            torch.cuda.synchronize()
+        configs["1_tiny"]["greedy_steps"] = {"steps": w1.steps, "B": 1, "dtype": "f32",
+                                             "us_per_step": a.elapsed_time(b) / w1.steps * 1e3,
+                                             "note": "mask in place, select, advance; launch latency bound"}
+        # workload 2: a regular expression's automaton (78 states) over 32,000 tokens
+        w2 = make_config(2)
+        t2 = [time_build(sd, nx, wl=w2) for sd, nx in ((fg.FSM_STATE_I32, True), (fg.FSM_STATE_U16, True),
+                                                       (fg.FSM_STATE_I32, False))]
+        configs["2_llama2_json"] = build_modes(
+            w2, *t2, rated=False,
+            why="2.5 M walks: a microsecond of work behind two launches, launch latency bound, not rated")
+        configs["3_llama3_random1k"] = build_modes(w, build_ms, u16_ms, maskonly_ms, rated=True)
+        # workload 4: 20,001 states x 152,064 tokens, 12.2 GB of int32 states
+        w4 = make_config(4)
+        t4 = [time_build(sd, nx, n=3, wl=w4) for sd, nx in ((fg.FSM_STATE_I32, True), (fg.FSM_STATE_U16, True),
+                                                            (fg.FSM_STATE_I32, False))]
+        configs["4_large_random20k"] = build_modes(
+            w4, *t4, rated=True,
+            why="the compressed table (2.6 MB) does not fit shared memory: look-ups beyond a row's own "
+                "table go through the read-only cache")
+        torch.cuda.empty_cache()
+    bound3, lpw3 = lookup_bound(w)
     walk_bytes = walks * 4 + w.Q * w.W * 4                    # next-state entries + bitmask words
     live_rows = w.B
     mask_bytes = live_rows * w.N * 2 * 2 + live_rows * w.W * 4
@@ -456,12 +581,12 @@ def run_ours(args):
                      "achieved": achieved, "peak": hbm_gbs, "unit": "GB/s",
                      "frac": achieved / hbm_gbs, "peak_kind": f"of {peak_kind}",
                      "algorithmic_bytes_per_launch": walk_bytes,
-                     "traffic": NCU_TRAFFIC.get("walk_sparse")},
+                     "traffic": ncu_traffic("walk_rows")},
         "roofline_mask_step": {"bound": "hbm", "kernel": "mask_step",
                                "achieved": mask_achieved, "peak": hbm_gbs, "unit": "GB/s",
                                "frac": mask_achieved / hbm_gbs, "peak_kind": f"of {peak_kind}",
                                "algorithmic_bytes_per_launch": mask_bytes,
-                               "traffic": NCU_TRAFFIC.get("mask_step")},
+                               "traffic": ncu_traffic("mask_step")},
         "roofline_sample_step": {"bound": "hbm", "kernel": "mask_step (categorical draw)",
                                  "achieved": mask_bytes / (sample_ms * 1e-3) / 1e9, "peak": hbm_gbs,
                                  "unit": "GB/s", "frac": mask_bytes / (sample_ms * 1e-3) / 1e9 / hbm_gbs,
@@ -475,27 +600,64 @@ def run_ours(args):
             "uint16_states": {"us": u16_ms * 1e3, "walks_per_s": walks / (u16_ms * 1e-3),
                               "hbm_write_bound_frac": (walks * 2.125 / (u16_ms * 1e-3) / 1e9) / hbm_gbs},
             "bitmask_only": {"us": maskonly_ms * 1e3, "walks_per_s": walks / (maskonly_ms * 1e-3),
-                             "smem_lookup_bound_frac": (walks / (maskonly_ms * 1e-3)) / SMEM_LOOKUP_BOUND,
-                             "note": "bound = 148 SMs x 32 lookups/clk x 1.965 GHz / 1.157 lookups "
-                                     "per walk (oracle-counted) = 8.04e12 walks/s"},
+                             "smem_lookup_bound_frac": (walks / (maskonly_ms * 1e-3)) / bound3,
+                             "note": f"bound = {sm_count} SMs x 32 lookups/clk x {sm_hz / 1e6:.0f} MHz "
+                                     f"(sampled under load) / {lpw3:.4f} lookups per walk (oracle-counted "
+                                     f"on a sample of states) = {bound3:.3e} walks/s"},
             "compressed_rows": {"us": csr_ms * 1e3, "walks_per_s": walks / (csr_ms * 1e-3),
                                 "entries": csr_nnz,
                                 "output_bytes": csr_nnz * 8 + (w.Q + 1) * 8 + w.Q * w.W * 4,
                                 "note": "fsm_index_build_csr: bitmask + per-state token lists with "
                                         "end states instead of the dense table"},
             "note": "whole builds (all launches), per-rank"},
+        "configs": configs,
+        "inputs_sha256": w.sha256(),
         "clocks": clocks,
         "e2e": {"value": walks * world / e2e_s, "unit": UNIT, "ms_per_step": e2e_s * 1e3,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "note": "host DFA, vocabulary, logits and states copied in, tokens/states/finished "
                         "copied out, every step; the index stays on the device for its consumer"},
-        "gpu_launches": 5 * args.steps,
+        "gpu_launches": LAUNCHES_PER_STEP * args.steps,
     }
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(w, starts)
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def run_only_build(args):
+    """A small case for profilers: builds workload K (optionally only the state slab
+    q0..q1-1, through fsm_index_build_rows) a few times and prints its time."""
+    import torch
+    import paper_2307_09702_b200 as fg
+    from paper_2307_09702_b200 import binding
+    from fsm_inputs import make_config
+    parts = args.only_build.split(":")
+    k = int(parts[0])
+    w = make_config(k)
+    d = w.dfa
+    q0, q1 = (int(parts[1]), int(parts[2])) if len(parts) == 3 else (0, d.Q)
+    torch.cuda.set_device(0)
+    fg.fsm_debug_set(binding.FSM_TUNE_WALK_ALGO, args.walk_algo)
+    modes = {"int32": (fg.FSM_STATE_I32, True), "uint16": (fg.FSM_STATE_U16, True),
+             "bitmask": (fg.FSM_STATE_I32, False)}
+    sd, want_next = modes[args.build_mode]
+    idx = fg.GuidedIndex(d.trans, d.accept, w.vocab_bytes, w.vocab_offsets, d.dead, w.eos_id, sd,
+                         want_next, q_begin=q0, q_end=q1)
+    for _ in range(args.warmup):
+        idx.build()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record()
+    for _ in range(args.steps):
+        idx.build()
+    b.record()
+    torch.cuda.synchronize()
+    assert int(idx.status.item()) == 0
+    us = a.elapsed_time(b) / args.steps * 1e3
+    print(json.dumps({"only_build": args.only_build, "mode": args.build_mode, "rows": q1 - q0, "N": w.N,
+                      "us": us, "walks_per_s": (q1 - q0) * w.N / (us * 1e-6)}))
 
 
 def main():
@@ -505,11 +667,20 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the per-workload block (workloads 1, 2 and 4)")
     ap.add_argument("--walk-algo", type=int, default=0, choices=[0, 1, 2, 3],
                     help="index walk: 0 automatic, 1 dense warp-tile, 2 row-wise work-avoiding, "
                          "3 bucket walk (bitmask-only builds)")
+    ap.add_argument("--only-build", default=None, metavar="K[:Q0:Q1]",
+                    help="profiling aid: only build workload K (or its state slab Q0..Q1-1) "
+                         "--steps times after --warmup builds")
+    ap.add_argument("--build-mode", default="int32", choices=["int32", "uint16", "bitmask"])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.only_build:
+        run_only_build(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:
