@@ -47,6 +47,9 @@ extern "C" {
 #define FSM_FLAG_WAIT_TIMEOUT 16 /* a bounded wait on an on-chip copy gave up; output invalid */
 #define FSM_FLAG_CSR_OVERFLOW 32 /* fsm_index_build_csr: more allowed pairs than `capacity`;
                                     row_offsets is complete, entries beyond capacity are missing */
+#define FSM_FLAG_INDEX 64        /* range-checked library only (built with -DFSM_CHECKED, file
+                                    name ending in _checked): an index computed from data was
+                                    outside its array; the access was skipped, output invalid */
 
 typedef enum { FSM_STATE_I32 = 0, FSM_STATE_U16 = 1 } fsm_state_dtype;
 typedef enum { FSM_LOGITS_F32 = 0, FSM_LOGITS_BF16 = 1 } fsm_logits_dtype;
@@ -292,6 +295,11 @@ int guided_step_csr(const void* logits_in, void* logits_out, int32_t logits_dtyp
                                        walk, 3 = bucket walk (bitmask-only builds; builds with
                                        a next-state table take 2).  Same results in every
                                        case */
+#define FSM_DEBUG_WAIT_PROBE 7      /* n > 0: once its table has arrived, a walk kernel waits
+                                       (at most n polls) for a completion that nothing will
+                                       ever signal, then takes its give-up path: it raises
+                                       FSM_FLAG_WAIT_TIMEOUT and returns.  For tests of that
+                                       path; the build's output is invalid while it is set */
 int fsm_debug_set(int32_t key, int32_t value);
 
 /*

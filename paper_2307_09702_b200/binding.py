@@ -17,9 +17,11 @@ FSM_LOGITS_F32, FSM_LOGITS_BF16 = 0, 1
 FSM_DEBUG_WEAK_HASH, FSM_TUNE_MASK_CLUSTER, FSM_TUNE_WALK_CTAS, FSM_TUNE_SMEM_TABLE_BYTES = 1, 2, 3, 4
 FSM_PROFILE_WALK = 5
 FSM_TUNE_WALK_ALGO = 6
+FSM_DEBUG_WAIT_PROBE = 7
 FSM_STATIC_SCRATCH_BYTES = 2 << 20
 FSM_FLAG_TRANS_RANGE, FSM_FLAG_OFFSETS, FSM_FLAG_STATE_RANGE = 1, 2, 4
 FSM_FLAG_CLASS_SPLIT, FSM_FLAG_WAIT_TIMEOUT = 8, 16
+FSM_FLAG_CSR_OVERFLOW, FSM_FLAG_INDEX = 32, 64
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libfsmguide.so")
@@ -33,6 +35,16 @@ class FsmError(RuntimeError):
 
 
 def library_path() -> str:
+    return _LIB_PATH
+
+
+def select_library(checked: bool) -> str:
+    """Switches every later call to the range-checked build of the library (``checked``) or
+    back to the regular one.  The two are separate images: knobs set through
+    ``fsm_debug_set`` belong to the library they were set in."""
+    global _lib, _LIB_PATH
+    _LIB_PATH = os.path.join(_PKG, "libfsmguide_checked.so" if checked else "libfsmguide.so")
+    _lib = None
     return _LIB_PATH
 
 

@@ -10,6 +10,10 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libfsmguide.so")
+# The same sources with -DFSM_CHECKED: every index that depends on data is range-checked
+# (FSM_FLAG_INDEX instead of a stray access).  A test aid, never the library the binding
+# loads by default.
+CHECKED_LIB_PATH = os.path.join(_PKG, "libfsmguide_checked.so")
 SOURCES = ["fsm_api.cu", "fsm_index.cu", "fsm_mask_step.cu"]
 # No --use_fast_math: the decode step compares logits as IEEE floats, subnormals included
 # (that flag flushes them to zero), and nothing on the path needs approximate division or
@@ -26,25 +30,30 @@ def _nvcc() -> str:
     raise RuntimeError("nvcc not found")
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB_PATH):
+def _stale(lib_path: str) -> bool:
+    if not os.path.exists(lib_path):
         return True
-    built = os.path.getmtime(LIB_PATH)
+    built = os.path.getmtime(lib_path)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(INCLUDE, "fsmguide.h")]
     return any(os.path.getmtime(d) > built for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compiles the library if it is missing or older than its sources."""
-    if not force and not _stale():
-        return LIB_PATH
-    tmp = LIB_PATH + f".tmp{os.getpid()}"
-    cmd = [_nvcc(), *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC, "-shared", "-o", tmp]
+def _compile(lib_path: str, extra: list[str], verbose: bool) -> None:
+    tmp = lib_path + f".tmp{os.getpid()}"
+    cmd = [_nvcc(), *NVCC_FLAGS, *extra, "-I", INCLUDE, "-I", CSRC, "-shared", "-o", tmp]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB_PATH)
+    os.replace(tmp, lib_path)
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Compiles the library, and its range-checked twin, if missing or older than the sources."""
+    if force or _stale(LIB_PATH):
+        _compile(LIB_PATH, [], verbose)
+    if force or _stale(CHECKED_LIB_PATH):
+        _compile(CHECKED_LIB_PATH, ["-DFSM_CHECKED"], verbose)
     return LIB_PATH
 
 

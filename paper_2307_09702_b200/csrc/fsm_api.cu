@@ -121,6 +121,7 @@ extern "C" int fsm_debug_set(int32_t key, int32_t value) {
         case FSM_TUNE_SMEM_TABLE_BYTES: slot = &t.smem_table_cap; break;
         case FSM_PROFILE_WALK: slot = &t.profile_walk; break;
         case FSM_TUNE_WALK_ALGO: slot = &t.walk_algo; break;
+        case FSM_DEBUG_WAIT_PROBE: slot = &t.wait_probe; break;
         default: return FSM_ERR_RANGE;
     }
     int old = *slot;

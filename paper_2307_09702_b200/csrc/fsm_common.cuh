@@ -22,6 +22,7 @@ struct Tunables {
     int smem_table_cap = 0;
     int profile_walk = 0;
     int walk_algo = 0;
+    int wait_probe = 0;
 };
 Tunables& tunables();
 
@@ -76,6 +77,28 @@ cudaError_t launch_cooperative(void (*kernel)(KArgs...), dim3 grid, dim3 block, 
 #ifdef __CUDACC__
 __device__ __forceinline__ void raise_flag(int32_t* status_word, int flag) {
     if (status_word != nullptr) atomicOr(status_word, flag);
+}
+
+// Range-checked build (-DFSM_CHECKED, a second library that is never the default): every
+// index that depends on data read from memory - a token id out of a sorted record, a state
+// out of a table, a position out of a counter - is compared with the size of the array it
+// goes into.  A violation raises FSM_FLAG_INDEX and the access is skipped; nothing traps.
+// In the regular build the test is constant-true and folds away.
+#ifdef FSM_CHECKED
+constexpr bool kChecked = true;
+#else
+constexpr bool kChecked = false;
+#endif
+
+template <typename I, typename B>
+__device__ __forceinline__ bool idx_ok(I i, B n, int32_t* status_word) {
+    if constexpr (kChecked) {
+        if (static_cast<long long>(i) < 0 || static_cast<long long>(i) >= static_cast<long long>(n)) {
+            raise_flag(status_word, FSM_FLAG_INDEX);
+            return false;
+        }
+    }
+    return true;
 }
 
 // ----------------------------------------------------------------------------

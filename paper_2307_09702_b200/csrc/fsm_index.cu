@@ -160,6 +160,7 @@ int build_rows_impl(const int32_t* dfa_trans, const uint8_t* accept, const uint8
     p.live = ws.live;
     p.row_order = row_order;
     p.chunk = kChunk;
+    p.wait_probe = tune.wait_probe;
     p.win_order = win_order;
     p.gstart = ws.gstart;
     p.count2 = ws.count2;

@@ -50,6 +50,7 @@ __device__ __forceinline__ bool stage_table(const WalkParams& p, TabT* stab, uin
     }
     bool ok = mbar_wait_bounded(bar, 0);
     if (!ok) ok = mbar_wait_bounded(bar, 0);  // drain before giving up
+    if (ok && p.wait_probe > 0) ok = mbar_wait_bounded(bar, 1, p.wait_probe);  // never completes
     if (!__syncthreads_and(ok)) {
         if (threadIdx.x == 0) raise_flag(p.status, FSM_FLAG_WAIT_TIMEOUT);
         return false;
@@ -91,13 +92,15 @@ __global__ void __launch_bounds__(kObThreads) mask_onebyte(const WalkParams p) {
         int nlive = 0;
         for (int k = 0; k * 32 < C; ++k) {
             const uint32_t m = __ldg(p.live + static_cast<size_t>(q) * 8 + k);
-            if ((m >> lane) & 1u) mine[nlive + __popc(m & ((1u << lane) - 1u))] = static_cast<uint8_t>(k * 32 + lane);
+            const int slot = nlive + __popc(m & ((1u << lane) - 1u));
+            if (((m >> lane) & 1u) && idx_ok(slot, 256, p.status)) mine[slot] = static_cast<uint8_t>(k * 32 + lane);
             nlive += __popc(m);
         }
         __syncwarp();
         // lane l holds words 4l .. 4l+3 of the block's 128
         uint4 acc = make_uint4(0, 0, 0, 0);
         const int wl = w0 + 4 * lane;
+        if (!idx_ok(nlive, 257, p.status)) nlive = 0;
         for (int j = 0; j < nlive; ++j) {
             const int c = mine[j];
             uint4 v;
@@ -143,6 +146,7 @@ __device__ __forceinline__ void bucket_tasks(const WalkParams& p, const TabT* __
                                              uint32_t Cs, const int32_t* s_gstart, int* s_next) {
     const uint32_t dead = p.dead;
     auto lookup = [&](uint32_t s, uint32_t c) -> uint32_t {
+        if (!idx_ok(static_cast<size_t>(s) * Cs + c, static_cast<size_t>(p.Q) * Cs, p.status)) return dead;
         if (FULL) return tab[s * Cs + c];
         return __ldg(tab + static_cast<size_t>(s) * Cs + c);
     };
@@ -164,13 +168,15 @@ __device__ __forceinline__ void bucket_tasks(const WalkParams& p, const TabT* __
         if (t >= ntasks) break;
         const int wat = static_cast<int>(t / parts);
         const int part = static_cast<int>(t - static_cast<int64_t>(wat) * parts);
-        const int win = p.win_order != nullptr ? __ldg(p.win_order + wat) : wat;
+        int win = p.win_order != nullptr ? __ldg(p.win_order + wat) : wat;
+        if (!idx_ok(win, nwin, p.status)) win = nwin;  // (nothing to walk there)
         const int pos = win * 32 + lane;
         uint4 rec = make_uint4(0, 0, 0, 0);
         int32_t id = -1;
-        if (pos < n_sorted) {
+        if (pos < n_sorted && idx_ok(pos, p.N, p.status)) {
             rec = __ldg(p.srec + pos);
             id = static_cast<int32_t>(rec.w);
+            if (!idx_ok(id, p.N, p.status)) id = -1;
         }
         const int len = rec.x & 0xFFu;
         const bool active = id >= 0 && len >= 2;
@@ -200,7 +206,8 @@ __device__ __forceinline__ void bucket_tasks(const WalkParams& p, const TabT* __
                     m &= m - 1;
                     const uint32_t s = __shfl_sync(kFullWarp, s2, l);
                     bool go = same && len > 2;
-                    uint32_t st = walk_rest<TabT, FULL, 2, kSortedInline>(tab, Cs, dead, rec, len, s, go);
+                    uint32_t st = walk_rest<TabT, FULL, 2, kSortedInline>(tab, Cs, dead, rec, len, s, go,
+                                                                          static_cast<uint32_t>(p.Q) * Cs, p.status);
                     if (go)  // longer than the record covers and still alive
                         st = raw_walk(p, st, p.vocab_offsets[id], p.vocab_offsets[id + 1], kSortedInline);
                     if (same && st != dead)

@@ -136,6 +136,7 @@ struct WalkParams {
     const int32_t* row_order;  // row-wise walk: rows in the order they are handed out, or null
     const int32_t* win_order;  // bucket walk: windows in the order they are handed out, or null
     int32_t chunk;             // dense walk: states per warp task (kChunk or kSmallChunk)
+    int32_t wait_probe;        // > 0: polls of a wait that nothing ends (test of the give-up path)
     // outputs
     uint32_t* mask;
     void* next;
@@ -227,20 +228,22 @@ __device__ __forceinline__ uint32_t raw_walk(const WalkParams& p, uint32_t s, in
 // (out-of-range entries were replaced by `dead` when the table was compressed), so the
 // shared-memory lookup needs no guard; the global-memory lookup is predicated to save
 // traffic.  On return `go` is true only for tokens longer than the record covers.
+// (`tab_n`: entries of the table, looked at by the range-checked build only.)
 template <typename TabT, bool FULL, int START, int END = kInlineBytes>
 __device__ __forceinline__ uint32_t walk_rest(const TabT* __restrict__ tab, uint32_t Cs,
                                               uint32_t dead, const uint4& tk, int len, uint32_t s,
-                                              bool& go) {
+                                              bool& go, uint32_t tab_n, int32_t* status) {
 #pragma unroll
     for (int i = START; i < END; ++i) {
         if (!__any_sync(kFullWarp, go)) break;
         const uint32_t c = tok_byte(tk, i);
         uint32_t ns;
         if (FULL) {
-            ns = tab[s * Cs + c];
+            ns = idx_ok(s * Cs + c, tab_n, status) ? tab[s * Cs + c] : dead;
         } else {
             ns = s;
-            if (go) ns = __ldg(tab + static_cast<size_t>(s) * Cs + c);
+            if (go && idx_ok(static_cast<size_t>(s) * Cs + c, tab_n, status))
+                ns = __ldg(tab + static_cast<size_t>(s) * Cs + c);
         }
         s = go ? ns : s;
         go = go && (ns != dead) && (i + 1 < len);

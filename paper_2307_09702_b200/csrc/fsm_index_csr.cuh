@@ -99,7 +99,10 @@ csr_scan(const int32_t* __restrict__ row_count, int32_t nrows, int64_t* __restri
         s_rank[threadIdx.x] = before + incl - mine;
     }
     __syncthreads();
-    for (int r = threadIdx.x; r < nrows; r += 1024) row_order[atomicAdd(&s_rank[bucket_of(r)], 1)] = r;
+    for (int r = threadIdx.x; r < nrows; r += 1024) {
+        const int at = atomicAdd(&s_rank[bucket_of(r)], 1);
+        if (idx_ok(at, nrows, status)) row_order[at] = r;
+    }
 }
 
 constexpr int kFillThreads = 128;
@@ -126,6 +129,7 @@ csr_fill(const WalkParams p, const uint16_t* __restrict__ tok_head,
     int2* longs = s_long[warp];
     for (int ri = blockIdx.x; ri < nrows; ri += gridDim.x) {
         const int r = row_order[ri];
+        if (!idx_ok(r, nrows, p.status)) continue;  // (block-uniform)
         const int q = p.q_begin + r;
         const uint32_t* mrow = p.mask + static_cast<size_t>(r) * p.G;
         const int32_t* trow = p.trans + static_cast<size_t>(q) * 256;
@@ -152,6 +156,7 @@ csr_fill(const WalkParams p, const uint16_t* __restrict__ tok_head,
         auto walk_longs = [&]() {
             for (int t = lane; t < nlong; t += 32) {
                 const int2 e = longs[t];
+                if (!idx_ok(e.y, p.N, p.status) || !idx_ok(row_at + e.x, capacity, p.status)) continue;
                 const uint32_t s = raw_walk(p, q, p.vocab_offsets[e.y], p.vocab_offsets[e.y + 1], 0);
                 csr_next[row_at + e.x] = static_cast<int32_t>(s);
             }
@@ -171,7 +176,8 @@ csr_fill(const WalkParams p, const uint16_t* __restrict__ tok_head,
             const int total = __shfl_sync(kFullWarp, incl, 31);
             int k = incl - cnt;
             while (bits) {
-                ids[k++] = static_cast<uint16_t>(lane * 32 + __ffs(bits) - 1);
+                if (idx_ok(k, 1024, p.status)) ids[k] = static_cast<uint16_t>(lane * 32 + __ffs(bits) - 1);
+                ++k;
                 bits &= bits - 1;
             }
             __syncwarp();
@@ -181,7 +187,7 @@ csr_fill(const WalkParams p, const uint16_t* __restrict__ tok_head,
                 const int j = j0 + lane;
                 bool walk = false;
                 int v = 0;
-                if (j < total) {
+                if (j < total && idx_ok(j, 1024, p.status) && idx_ok(base * 32 + ids[j], p.N, p.status)) {
                     v = base * 32 + ids[j];
                     uint32_t s = q;  // EOS keeps the state
                     if (dense_next != nullptr) {  // small automaton: the dense table was built
@@ -204,7 +210,8 @@ csr_fill(const WalkParams p, const uint16_t* __restrict__ tok_head,
                     __syncwarp();  // the entries other lanes set aside are visible to the walk
                     walk_longs();
                 }
-                if (walk) longs[nlong + __popc(m & ((1u << lane) - 1u))] = make_int2(at + j, v);
+                const int slot = nlong + __popc(m & ((1u << lane) - 1u));
+                if (walk && idx_ok(slot, kLongCap, p.status)) longs[slot] = make_int2(at + j, v);
                 nlong += __popc(m);
             }
             at += total;

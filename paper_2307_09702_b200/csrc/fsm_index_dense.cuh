@@ -32,14 +32,15 @@ __device__ __forceinline__ void walk_task(const WalkParams& p, const TabT* __res
     const bool multi = len > 1;
     const bool eos_lane = HAS_EOS && (v == p.eos_id);
     const bool store_ok = HAS_OUT && (v < p.N);
-    const TabT* f = first + (tk.x & 0xFFu);
+    const bool class_ok = idx_ok(tk.x & 0xFFu, Cs, p.status);  // (first byte's class: a column)
+    const TabT* f = first + (class_ok ? (tk.x & 0xFFu) : 0u);
     const size_t r0 = static_cast<size_t>(q0 - p.q_begin);
     OutT* outp = HAS_OUT ? static_cast<OutT*>(p.next) + r0 * p.N + v : nullptr;
     uint32_t* mp = p.mask + r0 * p.G + g;
     for (int j = 0; j < nq; ++j) {
-        uint32_t s = *f;
+        uint32_t s = class_ok ? static_cast<uint32_t>(*f) : dead;
         bool go = multi && (s != dead);
-        s = walk_rest<TabT, FULL, 1>(tab, Cs, dead, tk, len, s, go);
+        s = walk_rest<TabT, FULL, 1>(tab, Cs, dead, tk, len, s, go, static_cast<uint32_t>(p.Q) * Cs, p.status);
         if (go)  // longer than the inline record and still alive: finish on the raw bytes
             s = raw_walk(p, s, p.vocab_offsets[v], p.vocab_offsets[v + 1], kInlineBytes);
         if (HAS_EOS) {
@@ -124,6 +125,8 @@ __global__ void __launch_bounds__(kWalkThreads, 1) walk(const WalkParams p) {
             }
             bool ok = mbar_wait_bounded(&bar, parity);
             if (!ok) ok = mbar_wait_bounded(&bar, parity);  // drain before giving up
+            if (ok && p.wait_probe > 0)  // the phase after this one: nothing completes it
+                ok = mbar_wait_bounded(&bar, parity ^ 1, p.wait_probe);
             parity ^= 1;
             if (!__syncthreads_and(ok)) {
                 if (threadIdx.x == 0) raise_flag(p.status, FSM_FLAG_WAIT_TIMEOUT);

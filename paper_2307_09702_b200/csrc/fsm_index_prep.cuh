@@ -252,11 +252,12 @@ __device__ __forceinline__ void prepare_phase(
                 tok_head[v] = static_cast<uint16_t>(raw.b0 | (static_cast<uint32_t>(raw.len) << 8));
             if (tok_c1 != nullptr)  // (the array is padded to whole passes)
                 tok_c1[v] = static_cast<uint8_t>(t.len == 1 ? t.first : C);
-            if (t.len > 0) atomicAdd(&s_cnt[bucket_key(two, t.first, t.second_key)], 1);
+            const int key = bucket_key(two, t.first, t.second_key);
+            if (t.len > 0 && idx_ok(key, nkeys, status)) atomicAdd(&s_cnt[key], 1);
             if (planes != nullptr) {
                 const bool one = t.len == 1;
                 const uint32_t peers = __match_any_sync(kFullWarp, one ? t.first : 0xFFFF);
-                if (one && (tid & 31) == __ffs(peers) - 1)
+                if (one && (tid & 31) == __ffs(peers) - 1 && idx_ok(t.first, C, status) && idx_ok(v >> 5, Wp, status))
                     planes[static_cast<size_t>(t.first) * Wp + (v >> 5)] = peers;
             }
         }
@@ -285,7 +286,7 @@ __device__ __forceinline__ void sort_phase(
     const int32_t* count2, int32_t* cursor2, int32_t* __restrict__ start2, int32_t* __restrict__ gstart,
     uint4* __restrict__ srec, const uint32_t* live, int32_t q_begin, int32_t q_end, int32_t* row_order,
     int32_t* win_order, int* s_sort /* s_start[kKeysPad], s_cnt[kKeys] */, const TokenRaw& raw_first,
-    const uint8_t (&bytes_first)[kSortedInline]) {
+    const uint8_t (&bytes_first)[kSortedInline], int32_t* status) {
     int* s_start = s_sort;
     int* s_cnt = s_sort + kKeysPad;
     __shared__ int wsum[kPrepThreads / 32];
@@ -344,7 +345,7 @@ __device__ __forceinline__ void sort_phase(
         if (two) {
             for (int key = tid; key < kKeys; key += kPrepThreads) {
                 const int st = s_start[key], en = s_start[key + 1];
-                if (en > st && key % kKeyStride != 0) atomicAdd(&s_cnt[st >> 5], 1);
+                if (en > st && key % kKeyStride != 0 && idx_ok(st >> 5, nwin, status)) atomicAdd(&s_cnt[st >> 5], 1);
             }
         }
         __syncthreads();
@@ -360,7 +361,8 @@ __device__ __forceinline__ void sort_phase(
                 int base = 0;
                 if (lane == leader) base = atomicAdd(&s_hist[b], __popc(m));
                 base = __shfl_sync(kFullWarp, base, leader);
-                if (pass == 1 && w < nwin) win_order[base + __popc(m & ((1u << lane) - 1))] = w;
+                const int at = base + __popc(m & ((1u << lane) - 1));
+                if (pass == 1 && w < nwin && idx_ok(at, nwin, status)) win_order[at] = w;
             }
             __syncthreads();
             if (pass == 0 && tid == 0) {  // counts -> first positions
@@ -417,7 +419,10 @@ __device__ __forceinline__ void sort_phase(
         s_cnt[2 * tid] = front + inc2 - a0 - a1;
         s_cnt[2 * tid + 1] = front + inc2 - a1;
         __syncthreads();
-        for (int r = tid; r < nrows; r += kPrepThreads) row_order[atomicAdd(&s_cnt[bucket_of(r)], 1)] = r;
+        for (int r = tid; r < nrows; r += kPrepThreads) {
+            const int at = atomicAdd(&s_cnt[bucket_of(r)], 1);
+            if (idx_ok(at, nrows, status)) row_order[at] = r;
+        }
         return;
     }
     if (blockIdx.x == 0) {
@@ -445,7 +450,8 @@ __device__ __forceinline__ void sort_phase(
         const TokenInfo t = token_classify(raw, s_cls);
         const int key = t.len > 0 ? bucket_key(two, t.first, t.second_key) : 0;
         int rank = 0;
-        if (t.len > 0) rank = atomicAdd(&s_cnt[key], 1);
+        const bool placed = t.len > 0 && idx_ok(key, nkeys, status);
+        if (placed) rank = atomicAdd(&s_cnt[key], 1);
         uint8_t bytes[kSortedInline];
 #pragma unroll
         for (int i = 1; i < kSortedInline; ++i) {  // independent loads, issued together
@@ -476,7 +482,7 @@ __device__ __forceinline__ void sort_phase(
             }
         }
         __syncthreads();
-        if (t.len > 0) {
+        if (placed && idx_ok(s_cnt[key] + rank, N, status)) {
             const int pos = s_cnt[key] + rank;
             uint32_t w[3] = {static_cast<uint32_t>(min(t.len, kSortedInline + 1)), 0, 0};
             const int nb = min(t.len, kSortedInline);
@@ -557,7 +563,7 @@ __global__ void __launch_bounds__(kPrepThreads, 1) prepare_fused(const PrepParam
     grid.sync();
     sort_phase(a.vocab_bytes, a.vocab_offsets, a.vocab_nbytes, a.N, a.eos_id, a.meta, a.cls, a.count2,
                a.cursor2, a.start2, a.gstart, a.srec, a.live, a.q_begin, a.q_end, a.row_order, a.win_order,
-               s_dyn, raw_first, bytes_first);
+               s_dyn, raw_first, bytes_first, a.status);
 }
 
 }  // namespace

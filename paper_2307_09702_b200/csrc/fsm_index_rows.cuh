@@ -88,11 +88,12 @@ __device__ __forceinline__ void chunk_patch(const WalkParams& p, const TabT* __r
     const int len = rec.x & 0xFFu;
     const int32_t id = static_cast<int32_t>(rec.w);
     bool go = len > DEPTH;
-    uint32_t st = walk_rest<TabT, FULL, DEPTH, kSortedInline>(tab, Cs, dead, rec, len, s, go);
-    if (go)  // longer than the record covers and still alive: finish on the raw bytes
-        st = raw_walk(p, st, p.vocab_offsets[id], p.vocab_offsets[id + 1], kSortedInline);
+    uint32_t st = walk_rest<TabT, FULL, DEPTH, kSortedInline>(tab, Cs, dead, rec, len, s, go,
+                                                              static_cast<uint32_t>(p.Q) * Cs, p.status);
+    if (go && idx_ok(id, p.N, p.status))  // longer than the record covers and still alive:
+        st = raw_walk(p, st, p.vocab_offsets[id], p.vocab_offsets[id + 1], kSortedInline);  // the raw bytes
     // (a one-byte token of a one-level bucket already has its entry from the fill)
-    if (id >= 0 && len > 1 && st != dead) {
+    if (id >= 0 && len > 1 && st != dead && idx_ok(id, p.N, p.status)) {
         if (HAS_OUT) out.nrow[id] = static_cast<OutT>(st);
         atomicOr(out.mrow + (id >> 5), 1u << (id & 31));
     }
@@ -111,7 +112,7 @@ __device__ __forceinline__ void chunk_patch_level(const WalkParams& p, const Tab
 // The lane's record of a chunk (length 1 and id -1 beyond the chunk's end: nothing to walk).
 __device__ __forceinline__ uint4 chunk_fetch(const WalkParams& p, int pos, int count, int lane) {
     uint4 rec = make_uint4(1, 0, 0, 0xFFFFFFFFu);
-    if (lane < count) rec = __ldg(p.srec + pos + lane);
+    if (lane < count && idx_ok(pos + lane, p.N, p.status)) rec = __ldg(p.srec + pos + lane);
     return rec;
 }
 
@@ -127,6 +128,7 @@ __device__ __forceinline__ void visit_buckets(const WalkParams& p, const TabT* _
     const uint32_t dead = p.dead;
     const int lane = threadIdx.x & 31;
     auto lookup = [&](uint32_t s, uint32_t c) -> uint32_t {
+        if (!idx_ok(static_cast<size_t>(s) * Cs + c, static_cast<size_t>(p.Q) * Cs, p.status)) return dead;
         if (FULL) return tab[s * Cs + c];
         return __ldg(tab + static_cast<size_t>(s) * Cs + c);
     };
@@ -148,8 +150,9 @@ __device__ __forceinline__ void visit_buckets(const WalkParams& p, const TabT* _
         int at = 0;
 #pragma unroll
         for (int cb = 0; cb < 8; ++cb) {
-            if ((lm[cb] >> lane) & 1u)
-                ctx.cls[at + __popc(lm[cb] & ((1u << lane) - 1u))] = static_cast<uint8_t>(cb * 32 + lane);
+            const int slot = at + __popc(lm[cb] & ((1u << lane) - 1u));
+            if (((lm[cb] >> lane) & 1u) && idx_ok(slot, 256, p.status))
+                ctx.cls[slot] = static_cast<uint8_t>(cb * 32 + lane);
             at += __popc(lm[cb]);
         }
         if (lane == 0) *ctx.ncls = n_live;
@@ -182,12 +185,12 @@ __device__ __forceinline__ void visit_buckets(const WalkParams& p, const TabT* _
         uint32_t s2 = dead;
         if (two_level) {
             const int key2 = kb * 32 + lane;
-            if (key2 >= 1 && key2 <= C) {
+            if (key2 >= 1 && key2 <= C && idx_ok(c0 * kKeyStride + key2, kKeys, p.status)) {
                 cnt = __ldg(p.count2 + c0 * kKeyStride + key2);
                 start = __ldg(p.start2 + c0 * kKeyStride + key2);
                 s2 = lookup(s1, key2 - 1);
             }
-        } else if (lane == 0) {
+        } else if (lane == 0 && idx_ok(c0, 256, p.status)) {
             start = s_gstart[c0];
             cnt = s_gstart[c0 + 1] - start;
             s2 = s1;
@@ -221,11 +224,13 @@ __device__ __forceinline__ void visit_buckets(const WalkParams& p, const TabT* _
                 const int b_cnt = __shfl_sync(kFullWarp, cnt, l);
                 const uint32_t b_s = __shfl_sync(kFullWarp, s2, l);
                 for (int k = lane; k * 32 < b_cnt; k += 32)
-                    ctx.descs[b_at + k] = Desc<TabT>::pack(b_start + 32 * k, b_s, min(32, b_cnt - 32 * k));
+                    if (idx_ok(b_at + k, kRowDescCap, p.status))
+                        ctx.descs[b_at + k] = Desc<TabT>::pack(b_start + 32 * k, b_s, min(32, b_cnt - 32 * k));
             }
             if (nch <= 4)
                 for (int k = 0; k < nch; ++k)
-                    ctx.descs[at + k] = Desc<TabT>::pack(start + 32 * k, s2, min(32, cnt - 32 * k));
+                    if (idx_ok(at + k, kRowDescCap, p.status))
+                        ctx.descs[at + k] = Desc<TabT>::pack(start + 32 * k, s2, min(32, cnt - 32 * k));
         } else {
             uint32_t m = __ballot_sync(kFullWarp, alive);
             while (m) {
@@ -252,7 +257,8 @@ __device__ __forceinline__ void walk_chunk_list(const WalkParams& p, const TabT*
     using D = Desc<TabT>;
     constexpr int kPull = 2;
     const int lane = threadIdx.x & 31;
-    const int total = ctx.ctrs[1];
+    int total = ctx.ctrs[1];
+    if (!idx_ok(total, kRowDescCap + 1, p.status)) total = 0;
     while (true) {
         int i = 0;
         if (lane == 0) i = atomicAdd(&ctx.ctrs[2], kPull);
@@ -294,13 +300,15 @@ __device__ __forceinline__ void build_row_table(const TabT* __restrict__ tab, ui
 // Look-up of byte k (0..3) of a word of four packed class ids.
 template <bool REPL>
 __device__ __forceinline__ uint32_t lut_get(const uint8_t* lut_base, uint32_t lane_off,
-                                            uint32_t packed, int k) {
+                                            uint32_t packed, int k, int32_t* status) {
     if (REPL) {
         // byte 0 = lane_off (parity * 128 + lane * 4), byte 1 = class id: c * 256 + lane_off
         const uint32_t off = __byte_perm(packed, lane_off, 0x5504u | (static_cast<uint32_t>(k) << 4));
+        if (!idx_ok(off, kLutBytes - 3, status)) return 0;
         return *reinterpret_cast<const uint32_t*>(lut_base + off);
     }
     const uint32_t c = (packed >> (8 * k)) & 0xFFu;
+    if (!idx_ok(lane_off + c * 4, kLutBytes - 3, status)) return 0;
     return *reinterpret_cast<const uint32_t*>(lut_base + lane_off + c * 4);
 }
 
@@ -340,12 +348,12 @@ __device__ __forceinline__ void fill_row(const WalkParams& p, const uint8_t* lut
                 Vec32B o;
                 if constexpr (EPV == 8) {
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) o.w[k] = lut_get<REPL>(lut_base, lane_off, cc[u][k >> 2], k & 3);
+                    for (int k = 0; k < 8; ++k) o.w[k] = lut_get<REPL>(lut_base, lane_off, cc[u][k >> 2], k & 3, p.status);
                 } else {
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
-                        const uint32_t lo = lut_get<REPL>(lut_base, lane_off, cc[u][(2 * k) >> 2], (2 * k) & 3);
-                        const uint32_t hi = lut_get<REPL>(lut_base, lane_off, cc[u][(2 * k + 1) >> 2], (2 * k + 1) & 3);
+                        const uint32_t lo = lut_get<REPL>(lut_base, lane_off, cc[u][(2 * k) >> 2], (2 * k) & 3, p.status);
+                        const uint32_t hi = lut_get<REPL>(lut_base, lane_off, cc[u][(2 * k + 1) >> 2], (2 * k + 1) & 3, p.status);
                         o.w[k] = __byte_perm(lo, hi, 0x5410u);
                     }
                 }
@@ -356,8 +364,9 @@ __device__ __forceinline__ void fill_row(const WalkParams& p, const uint8_t* lut
     }
     // ragged tail, or a row that is not 32-byte aligned: entry by entry, still coalesced
     for (int v = done + threadIdx.x; v < p.N; v += kWalkThreads) {
-        const uint32_t c = c1[v];
-        nrow[v] = static_cast<OutT>(*reinterpret_cast<const uint32_t*>(lut_base + lane_off + c * (REPL ? 256 : 4)));
+        const uint32_t off = lane_off + c1[v] * (REPL ? 256 : 4);
+        if (idx_ok(off, kLutBytes - 3, p.status))
+            nrow[v] = static_cast<OutT>(*reinterpret_cast<const uint32_t*>(lut_base + off));
     }
 }
 
@@ -377,7 +386,8 @@ __device__ __forceinline__ void mask_row_from_planes(const WalkParams& p, const 
 #pragma unroll
             for (int u = 0; u < kBatch; ++u) {
                 v[u] = make_uint4(0, 0, 0, 0);
-                if (j0 + u < ncls) v[u] = __ldg(col + static_cast<size_t>(cls[j0 + u]) * (Gp / 4));
+                if (j0 + u < ncls && idx_ok(j0 + u, 256, p.status))
+                    v[u] = __ldg(col + static_cast<size_t>(cls[j0 + u]) * (Gp / 4));
             }
 #pragma unroll
             for (int u = 0; u < kBatch; ++u) {
@@ -482,6 +492,7 @@ __global__ void __launch_bounds__(kWalkThreads, 1) walk_rows(const WalkParams p,
         }
         bool ok = mbar_wait_bounded(&bar, 0);
         if (!ok) ok = mbar_wait_bounded(&bar, 0);  // drain before giving up
+        if (ok && p.wait_probe > 0) ok = mbar_wait_bounded(&bar, 1, p.wait_probe);  // never completes
         if (!__syncthreads_and(ok)) {
             if (threadIdx.x == 0) raise_flag(p.status, FSM_FLAG_WAIT_TIMEOUT);
             return;
@@ -517,7 +528,11 @@ __global__ void __launch_bounds__(kWalkThreads, 1) walk_rows(const WalkParams p,
     // Rows are taken in the order the preparation ranked them; position i of that order.
     // The CTA's first row has a fixed place; one thread draws the later ones, always one row
     // ahead (position and row number are on their way while a row is filled).
-    auto row_at = [&](int i) { return i >= nrows ? -1 : p.row_order != nullptr ? __ldg(p.row_order + i) : i; };
+    auto row_at = [&](int i) {
+        if (i >= nrows) return -1;
+        const int r = p.row_order != nullptr ? __ldg(p.row_order + i) : i;
+        return idx_ok(r, nrows, p.status) ? r : -1;
+    };
     int par = 0;
     int row = row_at(blockIdx.x);
     int at_next = 0;  // thread 0: position of the next row

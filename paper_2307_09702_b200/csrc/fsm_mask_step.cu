@@ -256,13 +256,14 @@ __device__ __forceinline__ void pool_vector(uint32_t bits, int first_id, const T
     const int total = __shfl_sync(kFullWarp, incl, 31);
     if (total == 0) return;
     int at = qn + incl - mine;
-    for (uint32_t todo = bits; todo != 0; todo &= todo - 1) q.id[at++] = first_id + __ffs(todo) - 1;
+    for (uint32_t todo = bits; todo != 0; todo &= todo - 1, ++at)
+        if (idx_ok(at, kQueue, p.status)) q.id[at] = first_id + __ffs(todo) - 1;
     qn += total;
     __syncwarp();
     int head = 0;
     for (; qn - head >= 32; head += 32) {
         const int id = q.id[head + lane];
-        take_better(best, gumbel_score(logit_of(in, id), id, row, p), id);
+        if (idx_ok(id, p.N, p.status)) take_better(best, gumbel_score(logit_of(in, id), id, row, p), id);
     }
     if (head > 0) {  // leftovers to the front
         const int rem = qn - head;
@@ -447,6 +448,9 @@ __global__ void __launch_bounds__(kStepThreads) mask_step(const StepParams p) {
         } else if (b.idx == p.eos_id) {
             p.finished[row] = 1;
             p.tokens[row] = b.idx;
+        } else if (!idx_ok(b.idx, p.N, p.status)) {
+            p.finished[row] = 2;  // (range-checked build only: a winner outside the vocabulary)
+            p.tokens[row] = -1;
         } else {
             p.tokens[row] = b.idx;
             if (p.csr_offsets != nullptr) {

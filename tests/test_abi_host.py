@@ -32,6 +32,20 @@ def test_every_declared_symbol_is_exported(fg):
         assert hasattr(fg, n), f"binding lacks {n}"
 
 
+def test_the_range_checked_library_is_built_and_exports_the_same_symbols(fg):
+    from paper_2307_09702_b200 import binding, build as b
+    assert os.path.exists(b.CHECKED_LIB_PATH) and b.CHECKED_LIB_PATH != fg.library_path()
+    L = ctypes.CDLL(b.CHECKED_LIB_PATH)
+    for n in declared_functions():
+        assert hasattr(L, n), n
+    try:
+        assert binding.select_library(True) == b.CHECKED_LIB_PATH
+        assert fg.fsm_debug_set(7, 5) == 0 and fg.fsm_debug_set(7, 0) == 5
+    finally:
+        binding.select_library(False)
+    assert fg.library_path().endswith("libfsmguide.so")
+
+
 def test_status_strings(fg):
     assert fg.fsm_status_string(0) == "FSM_OK"
     for code in range(-8, 0):
