@@ -16,6 +16,10 @@ whole step.  With N > 1 (torchrun) every rank runs the same-shaped workload on i
 GPU with its own automaton seed: the path shards over independent problems and
 has no data-path collective (weak scaling).
 
+``--shard states`` measures the other split instead: ONE workload-4 index (20,001 states
+x 152,064 tokens) divided over the ranks by state slabs, every rank building its slab with
+``fsm_index_build_rows`` and the slabs meeting in an NCCL all-gather (strong scaling).
+
 ``--impl reference`` times the CPU oracle on the host cores instead.
 """
 from __future__ import annotations
@@ -626,6 +630,160 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_sharded(args):
+    """`--shard states`: ONE index (workload 4: 20,001 states x 152,064 tokens, int32 states)
+    split over the ranks by state slabs.  A step = every rank builds its slab with
+    fsm_index_build_rows straight into its place in the full arrays, then the slabs meet in an
+    in-place NCCL all-gather (no kernel of this library is handed another rank's memory).
+    Strong scaling: the total work is fixed, `value` = Q*N / max-over-ranks step time."""
+    import torch
+    import paper_2307_09702_b200 as fg
+    from paper_2307_09702_b200 import binding, sharding
+    from fsm_inputs import make_config
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    if fg.fsm_device_check() != 0:
+        raise SystemExit("bench.py needs a compute-capability 10.x device")
+    fg.fsm_debug_set(binding.FSM_TUNE_WALK_ALGO, args.walk_algo)
+    w = make_config(4)
+    d = w.dfa
+    Q, N, W = d.Q, w.N, (w.N + 31) // 32
+    per = -(-Q // world)
+    q0, q1 = sharding.equal_slab(Q, rank, world)
+    pinned = lambda a, dt: torch.as_tensor(np.ascontiguousarray(a), dtype=dt).pin_memory()
+    h_trans, h_acc = pinned(d.trans, torch.int32), pinned(d.accept, torch.uint8)
+    h_vb, h_vo = pinned(w.vocab_bytes, torch.uint8), pinned(w.vocab_offsets, torch.int32)
+    d_trans, d_acc, d_vb, d_vo = (t.to(dev) for t in (h_trans, h_acc, h_vb, h_vo))
+    nbytes = int(w.vocab_offsets[-1])
+    full_mask = torch.zeros((world * per, W), dtype=torch.int32, device=dev)
+    full_next = torch.zeros((world * per, N), dtype=torch.int32, device=dev)
+    wsb = fg.fsm_index_workspace_bytes(Q, N, nbytes)
+    ws = torch.empty(wsb, dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    h_status = torch.zeros(1, dtype=torch.int32).pin_memory()
+
+    def build():
+        if q1 > q0:
+            rc = fg.fsm_index_build_rows(d_trans, d_acc, d_vb, d_vo, nbytes, Q, N, d.dead, w.eos_id, q0, q1,
+                                         full_mask[q0:q1], full_next[q0:q1], fg.FSM_STATE_I32, ws, wsb, status)
+            assert rc == 0, fg.fsm_status_string(rc)
+
+    def gather():
+        if dist is not None:
+            sharding.all_gather_slabs_in_place(full_mask, Q)
+            sharding.all_gather_slabs_in_place(full_next, Q)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        build()
+        gather()
+    barrier()
+    assert int(status.item()) == 0, "data-fault flag raised during warm-up"
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    fg.fsm_debug_set(binding.FSM_PROFILE_WALK, 1)
+    sampler = ClockSampler(local)
+    sampler.start()
+    barrier()
+    for i in range(args.steps):
+        ev[i][0].record()
+        build()
+        ev[i][1].record()
+        gather()
+        ev[i][2].record()
+    barrier()
+    clocks = sampler.stop()
+    fg.fsm_debug_set(binding.FSM_PROFILE_WALK, 0)
+    total_ms = ev[0][0].elapsed_time(ev[-1][2])
+    build_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
+    gather_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
+    walk = fg.fsm_profile_read()
+    walk_ms = float(np.mean(walk)) if walk else build_ms
+    # ---- end to end: the inputs come from pinned host memory and the status word goes back
+    e2e_steps = max(3, min(args.steps, 50))
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        d_trans.copy_(h_trans, non_blocking=True)
+        d_acc.copy_(h_acc, non_blocking=True)
+        d_vb.copy_(h_vb, non_blocking=True)
+        d_vo.copy_(h_vo, non_blocking=True)
+        build()
+        gather()
+        h_status.copy_(status, non_blocking=True)
+        torch.cuda.synchronize()
+    barrier()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+
+    def allmax(x):
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    total_ms, build_ms, gather_ms, walk_ms, e2e_s = map(allmax, (total_ms, build_ms, gather_ms, walk_ms, e2e_s))
+    # ---- every rank checks sampled rows of the gathered index (its own slab and the others')
+    # against the CPU oracle
+    from oracle import fsm_oracle
+    for q in sorted({0, q0, max(q0, q1 - 1), (q0 + 7919) % Q, Q - 1, (Q // 2 + 1000 * rank) % Q}):
+        m, n, _ = fsm_oracle.index_build(d.trans, d.accept, w.vocab_bytes, w.vocab_offsets, d.dead, w.eos_id,
+                                         q_begin=q, q_end=q + 1, threads=len(os.sched_getaffinity(0)))
+        assert (full_mask[q].cpu().numpy().view(np.uint32) == m[0]).all(), q
+        assert (full_next[q].cpu().numpy() == n[0]).all(), q
+    if rank != 0:
+        dist.destroy_process_group()
+        return
+    hbm_gbs, peak_kind = load_peaks()
+    walks = float(Q) * N
+    step_ms = total_ms / args.steps
+    slab_bytes = (q1 - q0) * (N * 4 + W * 4)
+    achieved = slab_bytes / (walk_ms * 1e-3) / 1e9
+    moved = (world - 1) * per * (N + W) * 4          # bytes every rank receives per step
+    h2d = sum(t.numel() * t.element_size() for t in (h_trans, h_acc, h_vb, h_vo))
+    line = {
+        "metric": METRIC, "value": walks / (step_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True,
+        "scaling": "strong", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "slab_build_us": build_ms * 1e3, "walk_kernel_us": walk_ms * 1e3, "allgather_us": gather_ms * 1e3,
+        "allgather_gbs_per_rank": (moved / (gather_ms * 1e-3) / 1e9) if world > 1 and gather_ms > 0 else None,
+        "config": {"workload": "4_large_random20k: ONE index, random DFA Q=20001 x Qwen2-shaped vocab "
+                               "N=152064, int32 next-state + packed bitmask, split over the ranks by "
+                               "state slabs and all-gathered (NCCL, in place)",
+                   "Q": Q, "N": N, "state_dtype": "int32", "shard": "states",
+                   "rows_per_rank": per, "parallelism": f"state slabs x{world} + all-gather",
+                   "l2": "outputs larger than L2: every rank writes its slab of the 12.2 GB index"},
+        "roofline": {"bound": "hbm", "kernel": "walk (index build: next-state + bitmask stores)",
+                     "achieved": achieved, "peak": hbm_gbs, "unit": "GB/s", "frac": achieved / hbm_gbs,
+                     "peak_kind": f"of {peak_kind}", "algorithmic_bytes_per_launch": slab_bytes,
+                     "traffic": None},
+        "inputs_sha256": w.sha256(),
+        "checked": "sampled rows of the gathered index equal the CPU oracle on every rank",
+        "clocks": clocks,
+        "e2e": {"value": walks / e2e_s, "unit": UNIT, "ms_per_step": e2e_s * 1e3,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 4,
+                "note": "automaton and vocabulary copied in from pinned host memory, status word "
+                        "copied out, every step; the index stays on the devices"},
+        "gpu_launches": 2 * args.steps,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
 def run_only_build(args):
     """A small case for profilers: builds workload K (optionally only the state slab
     q0..q1-1, through fsm_index_build_rows) a few times and prints its time."""
@@ -676,6 +834,9 @@ def main():
                     help="profiling aid: only build workload K (or its state slab Q0..Q1-1) "
                          "--steps times after --warmup builds")
     ap.add_argument("--build-mode", default="int32", choices=["int32", "uint16", "bitmask"])
+    ap.add_argument("--shard", default="none", choices=["none", "states"],
+                    help="states: split ONE workload-4 index over the ranks by state slabs and "
+                         "all-gather it (strong scaling) instead of one independent problem per rank")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.only_build:
@@ -683,6 +844,9 @@ def main():
         return
     if args.impl == "reference":
         run_reference(args)
+    elif args.shard == "states":
+        args.steps = min(args.steps, 300)      # a step writes 12.2 GB
+        run_sharded(args)
     else:
         run_ours(args)
 

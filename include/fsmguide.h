@@ -5,9 +5,10 @@
  *
  * C ABI.  Unless an argument is marked HOST, every array pointer is a DEVICE
  * pointer owned by the caller; the library neither allocates nor frees device
- * memory, never synchronises the stream and never aborts.  All work is
- * enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = the default
- * stream) and may still be running when a call returns.
+ * memory and never aborts.  The build and decode calls never synchronise the
+ * stream: all their work is enqueued on `cuda_stream` (a cudaStream_t passed as
+ * void*, NULL = the default stream) and may still be running when a call
+ * returns.  The index-file calls and fsm_profile_read block, and say so.
  *
  * Return value: FSM_OK, or a negative FSM_ERR_* code.  Errors that can be
  * detected from the scalar arguments and pointer values are returned before
@@ -36,6 +37,11 @@ extern "C" {
 #define FSM_ERR_RANGE (-6)     /* dead_state, eos_id or a row range is out of range */
 #define FSM_ERR_CUDA (-7)      /* a CUDA runtime call failed (launch, attribute) */
 #define FSM_ERR_DEVICE (-8)    /* no device of compute capability 10.x is current */
+#define FSM_ERR_IO (-9)        /* an index file cannot be opened, read or written, or is shorter
+                                  than its header says */
+#define FSM_ERR_FORMAT (-10)   /* not an index file of this version, a file for another problem
+                                  (sizes, dtype, dead/EOS ids or input digest differ from what
+                                  the caller expects), or its contents fail their checksum */
 
 /* Bits of *status_word (device int32). */
 #define FSM_FLAG_TRANS_RANGE 1   /* a transition outside [0,Q) was read; treated as dead */
@@ -275,6 +281,101 @@ int guided_step_csr(const void* logits_in, void* logits_out, int32_t logits_dtyp
                     int32_t sample,
                     float inv_temperature, uint64_t seed, uint64_t draw, int32_t* status_word,
                     void* cuda_stream);
+
+/*
+ * Index files (paper Section 3.2: the index is computed once per (automaton,
+ * vocabulary) pair and reused; the paper's example session switches such a
+ * cache off to time the build).  A built index - the bitmask with either the
+ * dense next-state table, no table, or the compressed rows - is written to one
+ * flat little-endian file and read back into device arrays the caller owns.
+ *
+ * File layout: a 128-byte header
+ *     bytes  0..7    "FSMGIDX1"
+ *            8..11   uint32 version (1)
+ *           12..15   int32  form          FSM_INDEX_DENSE | FSM_INDEX_BITMASK | FSM_INDEX_CSR
+ *           16..19   int32  Q
+ *           20..23   int32  N
+ *           24..27   int32  state_dtype   FSM_STATE_* of the dense table (0 otherwise)
+ *           28..31   int32  dead_state
+ *           32..35   int32  eos_id
+ *           36..39   (zero)
+ *           40..47   int64  nnz           entries of the compressed rows (0 otherwise)
+ *           48..55   uint64 payload_bytes
+ *           56..63   uint64 payload_check (see fsm_checksum64)
+ *           64..95   input_digest         32 bytes chosen by the caller, meant to be the
+ *                                         SHA-256 of the build's inputs (fsm_index_input_digest)
+ *           96..127  (zero)
+ * followed by the payload, arrays back to back, each padded with zeros to a
+ * multiple of 8 bytes: allowed_mask [Q*W] uint32; then for FSM_INDEX_DENSE
+ * next_state [Q*N] of state_dtype; for FSM_INDEX_CSR row_offsets [Q+1] int64,
+ * csr_tokens [nnz] int32, csr_next [nnz] int32.
+ *
+ * The three calls below are HOST-side: they block (they synchronise
+ * `cuda_stream` and wait for their own copies), stage the arrays through two
+ * pinned host buffers of 16 MiB that they allocate and free, and issue one
+ * cudaMemcpyAsync per staged piece.  `path` is a HOST string.  The array
+ * pointers in the descriptor are DEVICE pointers; arrays the form does not use
+ * are ignored.
+ */
+#define FSM_INDEX_DENSE 0   /* bitmask + next-state table */
+#define FSM_INDEX_BITMASK 1 /* bitmask only */
+#define FSM_INDEX_CSR 2     /* bitmask + compressed rows */
+
+typedef struct fsm_index_desc {
+    int32_t form;
+    int32_t Q, N;
+    int32_t state_dtype; /* FSM_INDEX_DENSE: FSM_STATE_I32 or FSM_STATE_U16 */
+    int32_t dead_state, eos_id;
+    int64_t nnz;         /* FSM_INDEX_CSR: entries of csr_tokens / csr_next (= row_offsets[Q]) */
+    uint8_t input_digest[32];
+    uint32_t* allowed_mask; /* [Q*W] */
+    void* next_state;       /* [Q*N] of state_dtype */
+    int64_t* row_offsets;   /* [Q+1] */
+    int32_t* csr_tokens;    /* [nnz] */
+    int32_t* csr_next;      /* [nnz] */
+} fsm_index_desc;
+
+/* Size in bytes of the file fsm_index_save writes for `desc` (sizes and form
+ * only; pointers are not looked at), or 0 when the descriptor is inconsistent. */
+size_t fsm_index_serialized_bytes(const fsm_index_desc* desc);
+
+/* Writes the index to `path` (replacing the file).  FSM_ERR_NULL / FSM_ERR_SHAPE /
+ * FSM_ERR_DTYPE / FSM_ERR_RANGE for a bad descriptor, FSM_ERR_IO when the file cannot
+ * be written, FSM_ERR_CUDA when a copy fails. */
+int fsm_index_save(const char* path, const fsm_index_desc* desc, void* cuda_stream);
+
+/* Reads the header of `path` into the scalar fields and input_digest of `*desc`
+ * (pointers are left alone), so that a caller can size its arrays.  Touches no
+ * device.  FSM_ERR_IO / FSM_ERR_FORMAT as above. */
+int fsm_index_peek(const char* path, fsm_index_desc* desc);
+
+/* Reads the index at `path` into the device arrays of `desc`.  Every scalar
+ * field of `desc` and its input_digest must equal the file's (an all-zero
+ * digest in `desc` accepts any): FSM_ERR_FORMAT otherwise, before any array is
+ * touched.  A file shorter than its header says gives FSM_ERR_IO; a payload
+ * that fails its checksum gives FSM_ERR_FORMAT after the arrays have been
+ * written - their contents are then invalid. */
+int fsm_index_load(const char* path, const fsm_index_desc* desc, void* cuda_stream);
+
+/* SHA-256 (FIPS 180-4) of `nbytes` HOST bytes into out32 (HOST, 32 bytes). */
+int fsm_sha256(const void* data, size_t nbytes, uint8_t* out32);
+
+/* The payload checksum of the index files, over HOST bytes (nbytes a multiple
+ * of 8): the wrap-around sum over 8-byte little-endian words w_i of
+ * mix(w_i + (i+1) * 0x9E3779B97F4A7C15), mix being the splitmix64 finaliser.
+ * Order-sensitive, cheap, not cryptographic: it catches truncation, bit rot
+ * and swapped blocks, nothing adversarial. */
+uint64_t fsm_checksum64(const void* data, size_t nbytes, uint64_t first_word_index);
+
+/* SHA-256 of the inputs of an index build, for the header's input_digest: the
+ * digest of the concatenation of the scalars (Q, N, dead_state, eos_id as int32,
+ * vocab_nbytes as int64, little-endian) and the DEVICE arrays dfa_trans [Q*256]
+ * int32, accept [Q] uint8, vocab_offsets [N+1] int32, vocab_bytes [vocab_nbytes].
+ * Blocks (copies the arrays to the host); out32 is a HOST pointer. */
+int fsm_index_input_digest(const int32_t* dfa_trans, const uint8_t* accept,
+                           const uint8_t* vocab_bytes, const int32_t* vocab_offsets,
+                           int64_t vocab_nbytes, int32_t Q, int32_t N, int32_t dead_state,
+                           int32_t eos_id, uint8_t* out32, void* cuda_stream);
 
 /*
  * Tuning and test hooks (no counterpart in the paper).  Sets a process-wide knob

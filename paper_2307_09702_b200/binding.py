@@ -22,6 +22,19 @@ FSM_STATIC_SCRATCH_BYTES = 2 << 20
 FSM_FLAG_TRANS_RANGE, FSM_FLAG_OFFSETS, FSM_FLAG_STATE_RANGE = 1, 2, 4
 FSM_FLAG_CLASS_SPLIT, FSM_FLAG_WAIT_TIMEOUT = 8, 16
 FSM_FLAG_CSR_OVERFLOW, FSM_FLAG_INDEX = 32, 64
+FSM_INDEX_DENSE, FSM_INDEX_BITMASK, FSM_INDEX_CSR = 0, 1, 2
+FSM_ERR_IO, FSM_ERR_FORMAT = -9, -10
+
+
+class IndexDesc(ctypes.Structure):
+    """``fsm_index_desc`` of the header, field for field."""
+    _fields_ = [("form", ctypes.c_int32), ("Q", ctypes.c_int32), ("N", ctypes.c_int32),
+                ("state_dtype", ctypes.c_int32), ("dead_state", ctypes.c_int32),
+                ("eos_id", ctypes.c_int32), ("nnz", ctypes.c_int64),
+                ("input_digest", ctypes.c_uint8 * 32),
+                ("allowed_mask", ctypes.c_void_p), ("next_state", ctypes.c_void_p),
+                ("row_offsets", ctypes.c_void_p), ("csr_tokens", ctypes.c_void_p),
+                ("csr_next", ctypes.c_void_p)]
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libfsmguide.so")
@@ -88,6 +101,21 @@ def lib() -> ctypes.CDLL:
                                       i32, i32, i32, ctypes.c_float, ctypes.c_uint64, ctypes.c_uint64,
                                       vp, vp]
         L.guided_step_csr.restype = ctypes.c_int
+        dp = ctypes.POINTER(IndexDesc)
+        L.fsm_index_serialized_bytes.argtypes = [dp]
+        L.fsm_index_serialized_bytes.restype = sz
+        L.fsm_index_save.argtypes = [ctypes.c_char_p, dp, vp]
+        L.fsm_index_save.restype = ctypes.c_int
+        L.fsm_index_peek.argtypes = [ctypes.c_char_p, dp]
+        L.fsm_index_peek.restype = ctypes.c_int
+        L.fsm_index_load.argtypes = [ctypes.c_char_p, dp, vp]
+        L.fsm_index_load.restype = ctypes.c_int
+        L.fsm_sha256.argtypes = [vp, sz, vp]
+        L.fsm_sha256.restype = ctypes.c_int
+        L.fsm_checksum64.argtypes = [vp, sz, ctypes.c_uint64]
+        L.fsm_checksum64.restype = ctypes.c_uint64
+        L.fsm_index_input_digest.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, i32, vp, vp]
+        L.fsm_index_input_digest.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -203,6 +231,60 @@ def guided_step_csr(logits_in, logits_out, logits_dtype, row_stride, states, fin
                                  _ptr(status_word), _stream(stream))
 
 
+def index_desc(form, Q, N, dead_state, eos_id, state_dtype=0, nnz=0, input_digest=None,
+               allowed_mask=None, next_state=None, row_offsets=None, csr_tokens=None,
+               csr_next=None) -> IndexDesc:
+    """Fills an ``fsm_index_desc`` (tensors become device pointers)."""
+    d = IndexDesc(form, Q, N, state_dtype, dead_state, eos_id, nnz)
+    if input_digest is not None:
+        ctypes.memmove(d.input_digest, bytes(input_digest), 32)
+    d.allowed_mask, d.next_state = _ptr(allowed_mask), _ptr(next_state)
+    d.row_offsets, d.csr_tokens, d.csr_next = _ptr(row_offsets), _ptr(csr_tokens), _ptr(csr_next)
+    return d
+
+
+def fsm_index_serialized_bytes(desc: IndexDesc) -> int:
+    return lib().fsm_index_serialized_bytes(ctypes.byref(desc))
+
+
+def fsm_index_save(path: str, desc: IndexDesc, stream=None) -> int:
+    return lib().fsm_index_save(os.fsencode(path), ctypes.byref(desc), _stream(stream))
+
+
+def fsm_index_peek(path: str, desc: IndexDesc) -> int:
+    return lib().fsm_index_peek(os.fsencode(path), ctypes.byref(desc))
+
+
+def fsm_index_load(path: str, desc: IndexDesc, stream=None) -> int:
+    return lib().fsm_index_load(os.fsencode(path), ctypes.byref(desc), _stream(stream))
+
+
+def fsm_sha256(data: bytes) -> bytes:
+    out = (ctypes.c_uint8 * 32)()
+    buf = ctypes.create_string_buffer(data, len(data)) if len(data) else None
+    rc = lib().fsm_sha256(ctypes.cast(buf, ctypes.c_void_p) if buf is not None else None, len(data),
+                          ctypes.cast(out, ctypes.c_void_p))
+    if rc != 0:
+        raise FsmError(rc, "fsm_sha256")
+    return bytes(out)
+
+
+def fsm_checksum64(data: bytes, first_word_index: int = 0) -> int:
+    buf = ctypes.create_string_buffer(data, len(data))
+    return lib().fsm_checksum64(ctypes.cast(buf, ctypes.c_void_p), len(data), first_word_index)
+
+
+def fsm_index_input_digest(dfa_trans, accept, vocab_bytes, vocab_offsets, vocab_nbytes, Q, N,
+                           dead_state, eos_id, stream=None) -> bytes:
+    out = (ctypes.c_uint8 * 32)()
+    rc = lib().fsm_index_input_digest(_ptr(dfa_trans), _ptr(accept), _ptr(vocab_bytes),
+                                      _ptr(vocab_offsets), vocab_nbytes, Q, N, dead_state, eos_id,
+                                      ctypes.cast(out, ctypes.c_void_p), _stream(stream))
+    if rc != 0:
+        raise FsmError(rc, "fsm_index_input_digest")
+    return bytes(out)
+
+
 class GuidedIndex:
     """Holds the device buffers of one vocabulary index and forwards to the C ABI.
 
@@ -241,6 +323,33 @@ class GuidedIndex:
                                   stream)
         if rc != 0:
             raise FsmError(rc, "fsm_index_build_rows")
+        return self
+
+    def _desc(self, digest) -> IndexDesc:
+        if (self.q_begin, self.q_end) != (0, self.Q):
+            raise ValueError("only a whole index is saved or loaded")
+        dense = self.next_state is not None
+        return index_desc(FSM_INDEX_DENSE if dense else FSM_INDEX_BITMASK, self.Q, self.N,
+                          self.dead_state, self.eos_id, self.state_dtype if dense else 0, 0, digest,
+                          self.allowed_mask, self.next_state)
+
+    def input_digest(self, stream=None) -> bytes:
+        return fsm_index_input_digest(self.trans, self.accept, self.vocab_bytes, self.vocab_offsets,
+                                      self.vocab_nbytes, self.Q, self.N, self.dead_state, self.eos_id,
+                                      stream)
+
+    def save(self, path: str, stream=None) -> None:
+        """Writes the built index to ``path`` (blocks)."""
+        rc = fsm_index_save(path, self._desc(self.input_digest(stream)), stream)
+        if rc != 0:
+            raise FsmError(rc, "fsm_index_save")
+
+    def load(self, path: str, stream=None) -> "GuidedIndex":
+        """Fills the index from a file saved for the same inputs instead of building it
+        (blocks); raises ``FsmError`` (``FSM_ERR_FORMAT``) when the file is for other inputs."""
+        rc = fsm_index_load(path, self._desc(self.input_digest(stream)), stream)
+        if rc != 0:
+            raise FsmError(rc, "fsm_index_load")
         return self
 
     def step(self, logits, states, finished, tokens_out, logits_out="inplace", stream=None):

@@ -101,6 +101,8 @@ extern "C" const char* fsm_status_string(int status) {
         case FSM_ERR_RANGE: return "FSM_ERR_RANGE: dead_state, eos_id, row range or key out of range";
         case FSM_ERR_CUDA: return "FSM_ERR_CUDA: a CUDA runtime call failed";
         case FSM_ERR_DEVICE: return "FSM_ERR_DEVICE: current device is not compute capability 10.x";
+        case FSM_ERR_IO: return "FSM_ERR_IO: index file cannot be opened, read or written, or is truncated";
+        case FSM_ERR_FORMAT: return "FSM_ERR_FORMAT: not an index file of this version, for another problem, or damaged";
         default: return "FSM_ERR_UNKNOWN";
     }
 }

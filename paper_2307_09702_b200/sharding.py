@@ -54,3 +54,26 @@ def all_gather_rows(local: torch.Tensor, total_rows: int, group=None) -> torch.T
     pieces = [torch.empty_like(padded) for _ in range(world)]
     dist.all_gather(pieces, padded.contiguous(), group=group)
     return torch.cat([pieces[r][: e - b] for r, (b, e) in enumerate(shards)], dim=0)
+
+
+def equal_slab(n: int, rank: int, world: int) -> tuple[int, int]:
+    """Rows ``[begin, end)`` of ``rank`` when every rank gets ``ceil(n / world)`` rows and the
+    last ranks take what is left (possibly nothing).  With slabs of one size the gathered
+    array is contiguous: row q of the whole sits at position q."""
+    per = -(-n // world)
+    begin = min(n, rank * per)
+    return begin, min(n, begin + per)
+
+
+def all_gather_slabs_in_place(full: torch.Tensor, total_rows: int, group=None) -> torch.Tensor:
+    """All-gather without staging copies.  ``full`` has ``world * ceil(total_rows / world)``
+    rows on every rank; rank r has written its ``equal_slab`` at its own position, and after
+    the call every rank holds all slabs (rows beyond ``total_rows`` are padding).  One
+    collective on tensors the ranks own; no kernel is handed another rank's memory."""
+    world = dist.get_world_size(group)
+    rank = dist.get_rank(group)
+    per = -(-total_rows // world)
+    if full.shape[0] != world * per:
+        raise ValueError("full must have world * ceil(total_rows / world) rows")
+    dist.all_gather_into_tensor(full, full[rank * per:(rank + 1) * per], group=group)
+    return full[:total_rows]

@@ -55,6 +55,13 @@ def _worker(rank, world, port, out_dir):
         st_ref, fin_ref = states.copy(), np.zeros(B, np.uint8)
         tok_ref, _ = fsm_oracle.mask_step(x, st_ref, fin_ref, rm, rn, d.dead, w.eos_id)
         assert (all_tok == tok_ref).all() and (all_st == st_ref).all()
+        # ---- equal slabs gathered in place (the layout of the sharded benchmark)
+        per = -(-d.Q // world)
+        full = torch.full((world * per, n.shape[1]), -5, dtype=torch.int32)
+        e0, e1 = sharding.equal_slab(d.Q, rank, world)
+        full[e0:e1] = torch.from_numpy(rn[e0:e1])
+        whole = sharding.all_gather_slabs_in_place(full, d.Q)
+        assert whole.shape[0] == d.Q and (whole.numpy() == rn).all()
         open(os.path.join(out_dir, f"ok{rank}"), "w").write("ok")
     finally:
         dist.destroy_process_group()
@@ -72,6 +79,13 @@ def test_contiguous_shards_cover_everything():
             assert max(sizes) - min(sizes) <= 1
     with pytest.raises(ValueError):
         sharding.contiguous_shards(5, 0)
+    for n in (0, 1, 5, 8, 1001, 20001):
+        for world in (1, 2, 3, 8):
+            slabs = [sharding.equal_slab(n, r, world) for r in range(world)]
+            per = -(-n // world)
+            assert slabs[0][0] == 0 and slabs[-1][1] == n
+            assert all(a[1] == b[0] for a, b in zip(slabs, slabs[1:]))
+            assert all(b == min(n, r * per) and e - b <= per for r, (b, e) in enumerate(slabs))
 
 
 def test_state_slabs_and_batch_slices_reassemble_with_gloo(tmp_path):
