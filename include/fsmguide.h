@@ -283,6 +283,35 @@ int guided_step_csr(const void* logits_in, void* logits_out, int32_t logits_dtyp
                     void* cuda_stream);
 
 /*
+ * Merging of identical index rows (paper Section 3: the index maps a state to its
+ * set of allowed tokens; Section 5: it is built from automata that are not
+ * reduced, so different states can carry the same row).
+ *
+ *   row_alias[q] = the smallest state whose row equals state q's, where "row" is
+ *   the bitmask row and, when next_state is given, also the next-state row (only
+ *   then can two states share one stored row of both arrays).  With next_state
+ *   NULL two states alias exactly when they allow the same set of tokens.
+ *
+ *   allowed_mask  [Q*W] as built, 4-byte aligned
+ *   next_state    [Q*N] of state_dtype as built, or NULL
+ *   row_alias     out, int32 [Q]; row_alias[q] <= q, row_alias[row_alias[q]] == row_alias[q]
+ *   n_unique      out, device int32: the number of distinct rows (states with row_alias[q] == q)
+ *   workspace     device scratch, 256-byte aligned, at least
+ *                 fsm_row_alias_workspace_bytes(Q) bytes (a few dozen bytes per state)
+ *
+ * Rows are grouped by a 64-bit hash and every merge is verified by comparing the
+ * two rows entry by entry, so the result does not depend on the hash (with
+ * FSM_DEBUG_WEAK_HASH set every row hashes alike and the result is the same).
+ * Three launches on `cuda_stream`; reads each row once, and rows that have an
+ * equal-hash partner a second time.
+ */
+size_t fsm_row_alias_workspace_bytes(int32_t Q);
+int fsm_index_row_alias(const uint32_t* allowed_mask, const void* next_state, int32_t state_dtype,
+                        int32_t Q, int32_t N, int32_t* row_alias, int32_t* n_unique,
+                        void* workspace, size_t workspace_bytes, int32_t* status_word,
+                        void* cuda_stream);
+
+/*
  * Index files (paper Section 3.2: the index is computed once per (automaton,
  * vocabulary) pair and reused; the paper's example session switches such a
  * cache off to time the build).  A built index - the bitmask with either the

@@ -101,6 +101,10 @@ def lib() -> ctypes.CDLL:
                                       i32, i32, i32, ctypes.c_float, ctypes.c_uint64, ctypes.c_uint64,
                                       vp, vp]
         L.guided_step_csr.restype = ctypes.c_int
+        L.fsm_row_alias_workspace_bytes.argtypes = [i32]
+        L.fsm_row_alias_workspace_bytes.restype = sz
+        L.fsm_index_row_alias.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, sz, vp, vp]
+        L.fsm_index_row_alias.restype = ctypes.c_int
         dp = ctypes.POINTER(IndexDesc)
         L.fsm_index_serialized_bytes.argtypes = [dp]
         L.fsm_index_serialized_bytes.restype = sz
@@ -229,6 +233,17 @@ def guided_step_csr(logits_in, logits_out, logits_dtype, row_stride, states, fin
                                  B, dead_state, eos_id, sample, inv_temperature,
                                  seed & 0xFFFFFFFFFFFFFFFF, draw & 0xFFFFFFFFFFFFFFFF,
                                  _ptr(status_word), _stream(stream))
+
+
+def fsm_row_alias_workspace_bytes(Q: int) -> int:
+    return lib().fsm_row_alias_workspace_bytes(Q)
+
+
+def fsm_index_row_alias(allowed_mask, next_state, state_dtype, Q, N, row_alias, n_unique, workspace,
+                        workspace_bytes, status_word=None, stream=None) -> int:
+    return lib().fsm_index_row_alias(_ptr(allowed_mask), _ptr(next_state), state_dtype, Q, N,
+                                     _ptr(row_alias), _ptr(n_unique), _ptr(workspace), workspace_bytes,
+                                     _ptr(status_word), _stream(stream))
 
 
 def index_desc(form, Q, N, dead_state, eos_id, state_dtype=0, nnz=0, input_digest=None,

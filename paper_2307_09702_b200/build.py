@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(_PKG, "libfsmguide.so")
 # (FSM_FLAG_INDEX instead of a stray access).  A test aid, never the library the binding
 # loads by default.
 CHECKED_LIB_PATH = os.path.join(_PKG, "libfsmguide_checked.so")
-SOURCES = ["fsm_api.cu", "fsm_index.cu", "fsm_index_io.cu", "fsm_mask_step.cu"]
+SOURCES = ["fsm_api.cu", "fsm_index.cu", "fsm_index_alias.cu", "fsm_index_io.cu", "fsm_mask_step.cu"]
 # No --use_fast_math: the decode step compares logits as IEEE floats, subnormals included
 # (that flag flushes them to zero), and nothing on the path needs approximate division or
 # transcendentals.
