@@ -48,19 +48,14 @@ AliasWorkspace carve_alias(void* base, int32_t Q) {
     return w;
 }
 
-__device__ __forceinline__ uint32_t mix32(uint32_t x) {
-    x ^= x >> 16;
-    x *= 0x7FEB352Du;
-    x ^= x >> 15;
-    x *= 0x846CA68Bu;
-    return x ^ (x >> 16);
-}
-
-// Contribution of value v at position i of a row.
+// Contribution of value v at position i of a row: one multiply-xorshift round keyed by the
+// position in the low half, the same value times an odd multiplier of the position in the
+// high half.  Cheap on purpose - the pass should run at the speed of its reads - and good
+// enough: every merge is verified entry by entry afterwards.
 __device__ __forceinline__ unsigned long long mix_at(uint32_t v, uint32_t i) {
-    const uint32_t a = mix32(v ^ (i * 0x9E3779B1u));
-    const uint32_t b = mix32(v + i * 0x85EBCA77u + 0x165667B1u);
-    return (static_cast<unsigned long long>(b) << 32) | a;
+    uint32_t x = (v ^ (i * 0x9E3779B1u)) * 0x85EBCA6Bu;
+    x ^= x >> 15;
+    return (static_cast<unsigned long long>(x * (2u * i + 1u)) << 32) + x;
 }
 
 // Sum of mix_at over row[0..n) for this thread's share; positions start at `base`.
